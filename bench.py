@@ -1,0 +1,328 @@
+"""Benchmark of the fused Tri-Accel optimizer pass.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is parameters per second of the whole job (N replicas), inputs
+resident in HBM; `e2e` is the same metric through ta_step_host with pinned HOST buffers
+(copies inside the timed region); `roofline` describes the dominant kernel (the update + cast
+kernel) against the measured HBM copy rate; `cpu_baseline` is the CPU checker timed on a
+bounded sample of the same workload.  `--impl reference` times the CPU checker alone.
+"""
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fused Tri-Accel step params/sec"
+UNIT = "params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernel_source_hash():
+    h = hashlib.sha256()
+    with open(os.path.join(ROOT, "paper_2508_16905_b200", "csrc", "kernels.cuh"), "rb") as f:
+        h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(kernel, workload, units):
+    """DRAM bytes per launch of `kernel` from the committed ncu capture, or None when there is no
+    capture for this workload or the kernel source changed since it was taken."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
+            rec = json.load(f)[kernel]
+    except Exception:
+        return None
+    if rec.get("kernels_cuh_sha256_16") != kernel_source_hash() or workload not in rec.get("valid_for", []):
+        return None
+    return rec["dram_bytes_per_param"] * units
+
+
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(wl, max_params):
+    """A run of whole layers of `wl` (after the first, to skip the embedding of the GPT workload when
+    it alone exceeds the budget) with at most max_params parameters."""
+    layers, total = [], 0
+    for l, (off, n) in enumerate(wl.table):
+        if n > max_params:
+            continue
+        if total + n > max_params:
+            break
+        layers.append(l)
+        total += n
+    return layers, total
+
+
+def time_oracle(wl, steps, warmup, budget_s, torch_device):
+    """Times the CPU checker, as it stands, on a bounded sample of layers; returns a dict."""
+    import numpy as np
+    import torch
+    from oracle import oracle as orc
+    from paper_2508_16905_b200 import workloads as W
+
+    # calibrate on a small sample, then size the sample so that all steps fit the budget
+    per_param_guess = 120e-9 * (1 + 0.5 * wl.num_probes) * (3.0 if wl.topk_ppm < 1000000 else 1.0)
+    max_params = int(max(2e5, min(wl.num_params, budget_s / max(1, steps + warmup) / per_param_guess)))
+    layers, n_sample = oracle_sample(wl, max_params)
+    if not layers:
+        layers, n_sample = [0], wl.table[0][1]
+    sub = [wl.table[l] for l in layers]
+    end = (sub[-1][0] + sub[-1][1] + 7) // 8 * 8
+    dev = torch_device
+    gen_total = wl.n_total
+
+    def host(t):
+        return t[:end].cpu().numpy() if t.dtype != torch.bfloat16 else t[:end].view(torch.int16).cpu().numpy().view(np.uint16)
+
+    w = host(W.make_weights(wl, dev)).copy()
+    D = host(W.make_curvature(wl, dev))
+    c = np.zeros(end, dtype=np.uint16)
+    o = orc.Oracle(sub, end, **wl.hparams())
+    times = []
+    for t in range(1, steps + warmup + 1):
+        g = host(W.make_grads(wl, t, dev))
+        hz = np.concatenate([D * orc.probe(wl.probe_seed, t, p, 0, end) for p in range(wl.num_probes)])
+        t0 = time.perf_counter()
+        o.step(w, g, hz, c, wl.probe_seed, t)
+        dt = time.perf_counter() - t0
+        if t > warmup:
+            times.append(dt)
+    del gen_total
+    sec = sum(times) / len(times)
+    return {"value": n_sample / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{len(layers)} layers ({n_sample} params) of {wl.name}, {len(times)} timed steps of the single-threaded C oracle",
+            "ms_per_step": sec * 1e3, "sample_params": n_sample}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import torch
+    from paper_2508_16905_b200 import workloads as W
+    wl = W.get(args.config)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    r = time_oracle(wl, steps, warmup, budget_s=150.0, torch_device=dev)
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "params": wl.num_params, "layers": len(wl.table), "sample": r["sample"]},
+            "cpu_baseline": {"value": r["value"], "unit": UNIT, "cores": 1, "kind": "oracle", "sample": r["sample"]},
+            "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def run_ours(args):
+    import torch
+    import paper_2508_16905_b200 as ta
+    from paper_2508_16905_b200 import dist as D
+    from paper_2508_16905_b200 import workloads as W
+
+    rank, local_rank, world = D.init("nccl")
+    torch.cuda.set_device(local_rank if world > 1 else 0)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    props = torch.cuda.get_device_properties(dev)
+    wl = W.get(args.config)
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    P, N = wl.num_probes, wl.n_total
+    l2_bytes = props.L2_cache_size
+
+    bytes_in_per_set = N * ((2 if wl.grad_dtype == "bf16" else 4) + 4 * P)
+    state_bytes = N * 6
+    # rotate over R buffer sets so that consecutive steps never find their inputs in L2
+    R = 1 if (bytes_in_per_set + state_bytes) > 4 * l2_bytes else max(2, -(-6 * l2_bytes // (bytes_in_per_set + state_bytes)))
+    h = ta.ta_create(wl.table, N, **wl.hparams())
+    curv = W.make_curvature(wl, dev)
+    sets = []
+    z = torch.empty(N, device=dev)
+    for r in range(R):
+        g = W.make_grads(wl, r + 1, dev)
+        hz = torch.empty(P * N, device=dev)
+        for p in range(P):
+            ta.ta_probe(h, wl.probe_seed, r + 1, p, z)
+            torch.mul(curv, z, out=hz[p * N:(p + 1) * N])
+        sets.append((W.make_weights(wl, dev), g, hz, torch.zeros(N, dtype=torch.int16, device=dev)))
+    del z, curv
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    def one_step(t):
+        w, g, hz, c = sets[t % R]
+        ta.ta_step(h, w, g, hz, c, wl.probe_seed, t)
+
+    t = 0
+    for _ in range(warmup):
+        t += 1
+        one_step(t)
+    torch.cuda.synchronize()
+    D.barrier()
+    sampler = ClockSampler(str(props.uuid) if str(props.uuid).startswith("GPU-") else "GPU-" + str(props.uuid)) if rank == 0 else None
+    launches0 = ta.ta_launch_count(h)
+    ta.ta_timing_begin(h, steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(steps):
+        t += 1
+        one_step(t)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    D.barrier()
+    ms_local = e0.elapsed_time(e1)
+    ms_sweep, ms_decide, ms_update, n_timed = ta.ta_timing_end(h)
+    launches = ta.ta_launch_count(h) - launches0
+    clocks = sampler.stop() if sampler else None
+    ms, units = D.aggregate(ms_local, wl.num_params * steps, device=dev)
+    stats, status = ta.ta_stats(h)
+    codes = [s.code for s in stats]
+    assert status.skipped == 0, "a benchmark step was skipped (non-finite synthetic input?)"
+
+    # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(steps, args.e2e_steps))
+        w_d, g_d, hz_d, c_d = sets[0]
+        wh, gh, hzh, ch = (x.cpu().pin_memory() for x in (w_d, g_d, hz_d, c_d))
+        h2 = ta.ta_create(wl.table, N, **wl.hparams())
+        ta.ta_step_host(h2, wh, gh, hzh, ch, wl.probe_seed, 1)          # warm-up: allocates the staging buffers
+        torch.cuda.synchronize()
+        D.barrier()
+        t0 = time.perf_counter()
+        for s in range(e2e_steps):
+            ta.ta_step_host(h2, wh, gh, hzh, ch, wl.probe_seed, 2 + s)
+        torch.cuda.synchronize()
+        dt_ms = (time.perf_counter() - t0) * 1e3
+        D.barrier()
+        codes2 = ta.ta_precision_codes(h2)
+        copy_params = sum(n for (_, n), cd in zip(wl.table, codes2) if cd < 2)
+        span = wl.table[-1][0] + wl.table[-1][1] - wl.table[0][0]
+        ms2, units2 = D.aggregate(dt_ms, wl.num_params * e2e_steps, device=dev)
+        e2e = {"value": units2 / (ms2 / 1e3), "unit": UNIT, "steps": e2e_steps, "ms_per_step": ms2 / e2e_steps,
+               "h2d_bytes_per_step": int(bytes_in_per_set + 4 * N), "d2h_bytes_per_step": int(4 * span + 2 * copy_params),
+               "api": "ta_step_host (pinned host tensors in, new weights and 16-bit copies out)"}
+        del wh, gh, hzh, ch
+        ta.ta_destroy(h2)
+
+    if rank != 0:
+        D.shutdown()
+        return 0
+
+    # ---- roofline of the dominant kernel (update + cast): algorithmic bytes / its measured duration
+    peak, peak_kind = measured_peak()
+    g_b = 2 if wl.grad_dtype == "bf16" else 4
+    copy_params = sum(n for (_, n), cd in zip(wl.table, codes) if cd < 2)
+    update_bytes = wl.num_params * (4 + g_b + 4) + 2 * copy_params
+    sweep_bytes = wl.num_params * (g_b + 4 * P)
+    upd_ms = ms_update / max(1, n_timed)
+    achieved = update_bytes / (upd_ms * 1e-3) / 1e9
+    step_bytes_min = wl.num_params * (4 + g_b + 4 * P + 4) + 2 * copy_params + (wl.num_params / 8 if wl.topk_ppm < 1000000 else 0)
+    ms_step = ms / steps
+    roofline = {"bound": "hbm", "kernel": "k_apply (master update + cast)", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                "traffic": recorded_traffic("k_apply", wl.name, wl.num_params),
+                "algorithmic_bytes_per_launch": update_bytes, "ms_per_launch": upd_ms,
+                "phases_ms_per_step": {"sweep": ms_sweep / max(1, n_timed), "decide_select": ms_decide / max(1, n_timed), "update": upd_ms},
+                "sweep_achieved_gbs": sweep_bytes / (ms_sweep / max(1, n_timed) * 1e-3) / 1e9,
+                "step": {"algorithmic_bytes": step_bytes_min, "achieved_gbs": step_bytes_min / (ms_step * 1e-3) / 1e9,
+                         "frac_of_peak": step_bytes_min / (ms_step * 1e-3) / 1e9 / peak,
+                         "frac_of_8tbs_nominal": step_bytes_min / (ms_step * 1e-3) / 1e9 / 8000.0}}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu = time_oracle(wl, steps=2, warmup=0, budget_s=20.0, torch_device=dev)
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    line = {"metric": METRIC, "value": units / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "params": wl.num_params, "layers": len(wl.table), "grad_dtype": wl.grad_dtype,
+                       "num_probes": P, "topk_ppm": wl.topk_ppm, "parallelism": f"replicas x{world}",
+                       "l2": (f"inputs of one step ({(bytes_in_per_set + state_bytes) / 1e6:.0f} MB) exceed L2 ({l2_bytes / 1e6:.0f} MB)"
+                              if R == 1 else f"{R} rotating buffer sets ({R * (bytes_in_per_set + state_bytes) / 1e6:.0f} MB) exceed L2 ({l2_bytes / 1e6:.0f} MB)"),
+                       "codes": {"fp16": codes.count(0), "bf16": codes.count(1), "fp32": codes.count(2)}},
+            "hbm_gbs_algorithmic": step_bytes_min / (ms_step * 1e-3) / 1e9,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+    print(json.dumps(line))
+    D.shutdown()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="gpt_1p3b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,245 @@
+/*
+ * triaccel.h -- C ABI of the Tri-Accel fused optimizer pass for NVIDIA B200 (sm_100a).
+ *
+ * One call of ta_step() runs, over every parameter tensor ("layer", a segment of one flat
+ * buffer), the per-step control-and-update pass of Tri-Accel (arXiv 2508.16905):
+ *   - per-layer gradient mean / variance and their exponential moving averages (Sec. 3.1),
+ *   - the sparse second-order signal: a Hutchinson diagonal estimate z*(Hz) from Rademacher
+ *     probes with a per-layer top-k magnitude mask (Abstract, Sec. 1, Sec. 3.2),
+ *   - the per-layer precision code FP16/BF16/FP32 from the variance EMA, with curvature
+ *     promotion, and the curvature-scaled step size (Sec. 3.1, Sec. 3.2, Sec. 3.4),
+ *   - the FP32 master-weight update fused with the cast into the layer's 16-bit copy
+ *     (Sec. 2 master-copy principle, Sec. 3.2 step size, Sec. 4.1 SGD).
+ * ta_batch_next() is the host-only memory-elastic batch rule (Sec. 3.3).
+ *
+ * Conventions
+ *   - Every function returns an int: TA_OK or a negative TA_ERR_* code.  Nothing throws.
+ *     ta_last_error() gives a static, human-readable string for the last failure of a handle.
+ *   - "device" pointers are CUDA device pointers of the handle's device; "host" pointers are
+ *     ordinary host memory.  The caller owns every buffer it passes.  The library owns the
+ *     handle, its per-layer state, its workspace and the mask bits; ta_destroy() frees them.
+ *   - All device work is enqueued on the stream passed in (a cudaStream_t cast to void*, NULL =
+ *     the default stream) and is asynchronous.  Only ta_stats(), ta_precision_codes(),
+ *     ta_step_host() and the state save/load calls wait for it.
+ *   - One handle belongs to one device (the device current at ta_create) and is not thread-safe.
+ *   - There is no CPU fallback: without a usable CUDA device ta_create fails with TA_ERR_CUDA.
+ *   - Flat-buffer layout: element i of layer l lives at flat index offset_l + i.  All flat
+ *     buffers (w, g, c, each probe of Hz, z_out) have n_total elements and use the same index.
+ *     Elements outside every segment ("gaps") are never read or written.
+ */
+#ifndef TRIACCEL_H
+#define TRIACCEL_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TA_OK          0
+#define TA_ERR_ARG    (-1)   /* NULL / out-of-range argument, invalid table or hyper-parameter      */
+#define TA_ERR_ALIGN  (-2)   /* a device pointer is not 16-byte aligned                             */
+#define TA_ERR_STATE  (-3)   /* call order: step did not increase, handle destroyed, size mismatch  */
+#define TA_ERR_CUDA   (-4)   /* a CUDA runtime call failed; ta_last_error() names it                */
+#define TA_ERR_NOMEM  (-5)   /* host or device allocation failed                                    */
+
+/* precision codes, in the order of the paper's case table (Sec. 3.1) */
+#define TA_CODE_FP16 0
+#define TA_CODE_BF16 1
+#define TA_CODE_FP32 2
+
+/* gradient element types */
+#define TA_GRAD_F32  0
+#define TA_GRAD_BF16 1
+
+#define TA_MAX_PROBES 8
+
+typedef struct ta_handle ta_handle;
+
+/* One layer: [offset, offset + length) in elements of the flat buffer. */
+typedef struct {
+    uint64_t offset;
+    uint64_t length;
+} ta_segment;
+
+/*
+ * Hyper-parameters.  struct_size must be sizeof(ta_hparams) of the header the caller compiled
+ * against (ABI growth).  Symbols follow the paper.
+ */
+typedef struct {
+    uint32_t struct_size;
+    float beta;          /* EMA smoothing, [0,1)                         Sec. 3.1 */
+    float tau_low;       /* v_l <  tau_low            -> FP16            Sec. 3.1 */
+    float tau_high;      /* v_l >= tau_high           -> FP32            Sec. 3.1 */
+    float tau_curv;      /* lambda_l > tau_curv  -> one level up         Sec. 3.2 */
+    float alpha;         /* eta_l = eta0 / (1 + alpha * lambda_l)        Sec. 3.2 */
+    float eta0;          /* base learning rate (see ta_set_lr)           Sec. 3.2 */
+    uint32_t topk_ppm;   /* mask keeps ceil(n_l * ppm / 1e6) (>= 1) largest |S|; 1000000 = dense */
+    uint32_t num_probes; /* P, one of 1, 2, 4, 8 */
+    uint32_t t_ctrl;     /* decisions are taken at steps with step % t_ctrl == 0   Sec. 3.4 */
+    uint32_t grad_dtype; /* TA_GRAD_F32 or TA_GRAD_BF16 */
+    float momentum;      /* must be 0 (plain SGD update) */
+    float weight_decay;  /* must be 0 */
+    uint32_t flags;      /* must be 0 */
+} ta_hparams;
+
+/* Per-layer statistics as of the last ta_step (host side, filled by ta_stats). */
+typedef struct {
+    float grad_mean;        /* mean of this step's gradient over the layer                      */
+    float grad_var;         /* population variance of this step's gradient over the layer       */
+    float ema_mean;         /* m_l                                                               */
+    float ema_var;          /* v_l                                                               */
+    float lambda_max;       /* max_i |S_i| / P, the curvature summary lambda_l                   */
+    float topk_threshold;   /* k-th largest |S_i| of the layer (S is the probe SUM, not the mean) */
+    float topk_mass;        /* sum of masked |S| / sum of all |S| (diagnostic)                   */
+    float eta_scale;        /* s_l = 1 / (1 + alpha * lambda_l), as of the last control step     */
+    uint64_t k;             /* mask population k_l                                               */
+    uint32_t code;          /* TA_CODE_*                                                         */
+    uint32_t near_threshold;/* 1 when v_l or lambda_l was within 1e-5 relative of a threshold at the last decision */
+} ta_layer_stats;
+
+typedef struct {
+    uint64_t step;                 /* step of the last ta_step                                  */
+    uint64_t nonfinite_count;      /* non-finite values seen in g and Hz at that step           */
+    uint32_t skipped;              /* 1: that step changed nothing because of non-finite input  */
+    uint32_t near_threshold_count; /* layers flagged near_threshold at the last decision        */
+} ta_step_status;
+
+/*
+ * ta_create -- validates the segment table and hyper-parameters, plans the sweep and allocates
+ * the library-owned device state on the current device.
+ *   table    host, L entries, ascending and non-overlapping, every length in [1, 2^32 - 2];
+ *            gaps between segments are allowed.  Offsets that are multiples of 4 elements give
+ *            fully vectorised access; any offset is handled correctly.
+ *   n_total  elements of every flat buffer; >= last offset + length; a multiple of 4.
+ *   hp       host; see ta_hparams.
+ *   out      receives the handle.
+ * Initial state (Sec. 3.1): m_l = v_l = 0, lambda_l = 0, s_l = 1, code BF16 (the default mode),
+ * mask empty.  Errors: TA_ERR_ARG, TA_ERR_NOMEM, TA_ERR_CUDA; *out is NULL on error.
+ */
+int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hparams *hp, ta_handle **out);
+
+/* Frees the handle and everything it owns.  NULL is allowed. */
+int ta_destroy(ta_handle *h);
+
+/*
+ * ta_step -- one optimizer pass (asynchronous).
+ *   w      device float[n_total], FP32 master weights, updated in place:
+ *          w_i <- fl32(w_i - eta_l * g_i), eta_l = fl32(eta0 * s_l)                  (Sec. 3.2, 4.1)
+ *   g      device, float[n_total] or bfloat16[n_total] per hp.grad_dtype; read only
+ *   Hz     device float[P][n_total] (probe p at Hz + p * n_total), the caller's products
+ *          H z^(p) with z^(p) = the probe ta_probe() writes for (probe_seed, step, p); or NULL,
+ *          in which case lambda_l, the threshold and the mask of the last step with Hz are kept
+ *          (Sec. 3.2: curvature only every T iterations)
+ *   c      device uint16[n_total], the 16-bit working copy: for layers coded FP16 / BF16 the
+ *          round-to-nearest-even cast of the new w (IEEE binary16 with subnormals and overflow to
+ *          inf / bfloat16); layers coded FP32 are left untouched                       (Sec. 2)
+ *   probe_seed, step   key the Rademacher generator; step must be larger than at the previous
+ *          call and below 2^32; decisions are taken when step % t_ctrl == 0, held otherwise.
+ * If any gradient or Hz value inside a segment is not finite, the whole step changes nothing
+ * (weights, copies, per-layer state) and ta_stats reports skipped = 1.
+ * Errors: TA_ERR_ARG (NULL w/g/c), TA_ERR_ALIGN (a pointer not 16-byte aligned), TA_ERR_STATE
+ * (step not increasing), TA_ERR_CUDA.  On error nothing is enqueued.
+ */
+int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
+            uint64_t probe_seed, uint64_t step, void *stream);
+
+/*
+ * ta_step_host -- the same pass for callers whose tensors live in HOST memory (ideally pinned).
+ * Copies w, g and Hz to library-owned device staging buffers (allocated at the first call, kept
+ * until ta_destroy), runs ta_step, waits, then copies back the new w of every layer and the new c
+ * of the layers coded FP16 / BF16 (c_host of FP32-coded layers and of gaps is left untouched; a
+ * skipped step copies nothing back).  Returns after the stream has drained.
+ * Arguments as for ta_step, but all four buffers are host pointers.  Errors as ta_step, plus
+ * TA_ERR_NOMEM when the staging buffers cannot be allocated.
+ */
+int ta_step_host(ta_handle *h, float *w_host, const void *g_host, const float *Hz_host, uint16_t *c_host,
+                 uint64_t probe_seed, uint64_t step, void *stream);
+
+/* Sets eta0 for the following steps; the caller owns warm-up and decay schedules (Sec. 4.3). */
+int ta_set_lr(ta_handle *h, float eta0);
+
+/*
+ * ta_probe -- writes the Rademacher probe z^(p) of (probe_seed, step), +1.0f / -1.0f, for all
+ * n_total flat elements to z_out (device float[n_total], 16-byte aligned).  These are the signs
+ * the sweep regenerates in registers.  The generator is Philox-4x32 with 10 rounds (Salmon et al.,
+ * SC'11): for flat element i, with block = i / 4096, r = i % 4096, row = r / 128,
+ * slot = (r / 4) % 32, comp = r % 4, the sign bit is bit (4*row + comp) of the 128-bit output of
+ * Philox(counter = (q_lo, q_hi, step, p), key = (seed_lo, seed_hi)), q = 32*block + slot;
+ * z = +1 for a 0 bit, -1 for a 1 bit.  p < num_probes.
+ */
+int ta_probe(ta_handle *h, uint64_t probe_seed, uint64_t step, uint32_t p, float *z_out, void *stream);
+
+/*
+ * ta_stats -- waits for the stream of the last ta_step, then fills out_host[L] and *status
+ * (either may be NULL).  Step (1) of the control loop of Sec. 3.4.
+ */
+int ta_stats(ta_handle *h, ta_layer_stats *out_host, ta_step_status *status);
+
+/* ta_precision_codes -- waits like ta_stats, then writes the L current codes (TA_CODE_*). Sec. 3.1 */
+int ta_precision_codes(ta_handle *h, uint8_t *out_host);
+
+/*
+ * ta_masks -- the top-k mask of the last step with Hz: bit (i & 31) of word i >> 5 is set when
+ * flat element i is among the k_l largest |S| of its layer (ties: lower index first); bits of
+ * gaps are 0.  *dev_bits is library-owned device memory, valid until the next ta_step with Hz or
+ * ta_destroy; read it on the stream used for ta_step.  With topk_ppm == 1000000 every element is
+ * in the mask, nothing is stored, and *dev_bits = NULL, *num_words = 0.
+ */
+int ta_masks(ta_handle *h, const uint32_t **dev_bits, uint64_t *num_words);
+
+/* Number of kernels the library launched on behalf of this handle so far (for benchmarks). */
+int ta_launch_count(ta_handle *h, uint64_t *count);
+
+/*
+ * Per-phase device timing (a measurement aid).  After ta_timing_begin(h, n) the next n calls of
+ * ta_step record CUDA events on their stream before the sweep, after it, after the decisions
+ * (including the top-k selection) and after the update.  ta_timing_end waits for the stream and
+ * returns the summed milliseconds of the three phases and the number of steps they cover.
+ */
+int ta_timing_begin(ta_handle *h, uint32_t max_steps);
+int ta_timing_end(ta_handle *h, double *ms_sweep, double *ms_decide, double *ms_update, uint32_t *steps);
+
+/* Static description of the last error of this handle ("" if none).  h may be NULL: then the
+ * last ta_create failure of the calling thread. */
+const char *ta_last_error(const ta_handle *h);
+
+/*
+ * Per-layer state checkpoint: EMAs, lambda, threshold, codes, step scale, mask bits, last step.
+ * ta_state_size gives the byte count; ta_state_save writes it to a host buffer (waits for the
+ * stream); ta_state_load restores it into a handle created with the same table and
+ * hyper-parameters (TA_ERR_STATE otherwise).  The next step after a load is bit-identical to
+ * the one the saved handle would have taken.
+ */
+int ta_state_size(ta_handle *h, uint64_t *bytes);
+int ta_state_save(ta_handle *h, void *buf_host, uint64_t bytes);
+int ta_state_load(ta_handle *h, const void *buf_host, uint64_t bytes);
+
+/*
+ * Memory-elastic batch rule (Sec. 3.3), host only:
+ *   B <- B + delta_up    if MemUsage <  rho_low  * MemMax
+ *   B <- B - delta_down  if MemUsage >  rho_high * MemMax
+ *   B unchanged otherwise; the result is clamped to [B_min, B_max] and stored back in bc->B.
+ * mem_reader(user, &free_bytes, &total_bytes) returns 0 on success; NULL selects cudaMemGetInfo
+ * of the current device.  MemUsage = total - free; MemMax = mem_budget_bytes if non-zero, else
+ * total.  Errors: TA_ERR_ARG (NULL, rho_low > rho_high, B_min > B_max, negative deltas),
+ * TA_ERR_CUDA (the reader failed; B is left unchanged).
+ */
+typedef int (*ta_mem_reader)(void *user, uint64_t *free_bytes, uint64_t *total_bytes);
+
+typedef struct {
+    int64_t B;
+    int64_t delta_up, delta_down;
+    int64_t B_min, B_max;
+    double rho_low, rho_high;
+    uint64_t mem_budget_bytes;
+    ta_mem_reader mem_reader;
+    void *user;
+} ta_batch_ctrl;
+
+int ta_batch_next(ta_batch_ctrl *bc, int64_t *B_next);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRIACCEL_H */

@@ -1,0 +1,877 @@
+// Device code of the Tri-Accel optimizer pass for sm_100a.
+//
+// The flat parameter buffer is cut into "rows" of 128 consecutive elements on a global grid
+// (row r covers flat indices [128 r, 128 r + 128)).  A warp reads one row per instruction:
+// lane j owns the four elements 128 r + 4 j .. + 3, i.e. one 16-byte vector of a float buffer.
+// 32 rows make a 4096-element block; the Rademacher bits of lane j for a whole block come from
+// one Philox call, so a lane pays one generator call per 128 elements it touches.
+//
+// Work is described by "items": a contiguous piece of ONE layer, handled by one warp.  Items are
+// cut on the global row grid, so only the first and last row of a layer can be partial; partial
+// rows take a scalar path with per-element bounds checks.  Gaps between layers are never touched.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ta {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr uint32_t kNonFiniteBits = 0x7F800000u;   // |x| bit patterns at or above this are inf / NaN
+constexpr int kHistBins = 2048;                    // radix-select levels: 11 + 11 + 9 bits of |S|
+
+struct Item {
+    uint64_t begin;   // first flat element
+    uint32_t len;     // elements, all inside layer `seg`
+    uint32_t seg;
+};
+
+// Per-layer state kept on the device between steps.
+struct LayerState {
+    double grad_mean, grad_var, topk_mass;
+    float ema_mean, ema_var;        // m_l, v_l                     (Sec. 3.1)
+    float lambda_max, thr;          // max|S|/P, k-th largest |S|   (Sec. 3.2)
+    float eta_scale, eta;           // s_l, eta_l = eta0 * s_l      (Sec. 3.2)
+    uint32_t code, near;            // precision code               (Sec. 3.1)
+};
+
+// Per-layer results of one sweep, before the decision to commit or skip the step.
+struct LayerScratch {
+    double mean, var, sum_abs;
+    unsigned long long bad;
+    uint32_t amax, amin;
+};
+
+struct Status {
+    unsigned long long step, nonfinite;
+    uint32_t skipped, near_count;
+    uint32_t done_counter, pad;
+};
+
+// Per-layer bookkeeping of the radix select.
+struct SelectState {
+    uint32_t prefix;      // bits of the threshold fixed so far
+    uint32_t remaining;   // how many elements are still to be taken inside the prefix
+    uint32_t thr_bits;    // final threshold bit pattern
+    uint32_t take_equal;  // how many elements equal to the threshold belong to the mask
+    uint32_t surplus;     // 1: more elements equal the threshold than are taken (index tie-break needed)
+    uint32_t pad;
+};
+
+struct Hyper {
+    float beta, tau_low, tau_high, tau_curv, alpha;
+    uint32_t num_probes, t_ctrl, topk_ppm;
+};
+
+// ------------------------------------------------------------------ Philox-4x32-10
+
+// Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3" (SC'11).
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Bits of lane `slot` for the 4096-element block `block`: 128 bits, bit 4*row + comp.
+__device__ __forceinline__ void probe_bits(uint64_t block, uint32_t slot, uint64_t seed, uint32_t step,
+                                           uint32_t p, uint32_t (&out)[4])
+{
+    const uint64_t q = block * 32ull + slot;
+    philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), step, p, (uint32_t)seed, (uint32_t)(seed >> 32), out);
+}
+
+__device__ __forceinline__ uint32_t pick_word(const uint32_t (&x)[4], uint32_t j)
+{
+    uint32_t lo = (j & 1u) ? x[1] : x[0];
+    uint32_t hi = (j & 1u) ? x[3] : x[2];
+    return (j & 2u) ? hi : lo;
+}
+
+// ------------------------------------------------------------------ small helpers
+
+__device__ __forceinline__ float4 ld_stream(const float *p)
+{
+    return __ldcs(reinterpret_cast<const float4 *>(p));
+}
+__device__ __forceinline__ float4 ld_keep(const float *p)
+{
+    return __ldg(reinterpret_cast<const float4 *>(p));
+}
+
+template <bool BF16> struct GradVec;
+template <> struct GradVec<false> {
+    static __device__ __forceinline__ float4 load4(const void *g, uint64_t i, bool stream)
+    {
+        const float *p = static_cast<const float *>(g) + i;
+        return stream ? ld_stream(p) : ld_keep(p);
+    }
+    static __device__ __forceinline__ float load1(const void *g, uint64_t i)
+    {
+        return __ldg(static_cast<const float *>(g) + i);
+    }
+};
+template <> struct GradVec<true> {
+    static __device__ __forceinline__ float4 load4(const void *g, uint64_t i, bool stream)
+    {
+        const uint2 *p = reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(g) + i);
+        const uint2 v = stream ? __ldcs(p) : __ldg(p);
+        float4 r;
+        r.x = __uint_as_float(v.x << 16);
+        r.y = __uint_as_float(v.x & 0xFFFF0000u);
+        r.z = __uint_as_float(v.y << 16);
+        r.w = __uint_as_float(v.y & 0xFFFF0000u);
+        return r;
+    }
+    static __device__ __forceinline__ float load1(const void *g, uint64_t i)
+    {
+        return __uint_as_float((uint32_t)__ldg(static_cast<const uint16_t *>(g) + i) << 16);
+    }
+};
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Sum over a 256-thread block in a fixed order; result valid in every thread.
+__device__ __forceinline__ double block_sum(double v, double *smem /*[kWarps]*/)
+{
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) smem[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += smem[w];
+    return t;
+}
+
+// ------------------------------------------------------------------ phase A: the sweep
+
+struct SweepArgs {
+    const Item *items;
+    uint32_t n_items, n_batches;
+    const void *g;
+    const float *hz;          // [P][n_total] or unused when P == 0
+    uint64_t n_total;
+    uint64_t seed;
+    uint32_t step;
+    // per-item partial results
+    double *p_s1, *p_s2, *p_sa;
+    uint32_t *p_amax, *p_amin, *p_bad;
+    // top-k only
+    float *abs_s;             // [n_total] |S|
+    uint32_t *hist;           // [L][kHistBins], level-1 histogram of |S| bit patterns
+};
+
+template <int P> struct RowData {
+    float4 g;
+    float4 hz[P > 0 ? P : 1];
+};
+
+// Balanced pairwise sum: adjacent pairs, level by level.
+template <int P> __device__ __forceinline__ float pairwise(const float (&t)[P > 0 ? P : 1])
+{
+    if constexpr (P == 2) {
+        return __fadd_rn(t[0], t[1]);
+    } else if constexpr (P == 4) {
+        return __fadd_rn(__fadd_rn(t[0], t[1]), __fadd_rn(t[2], t[3]));
+    } else if constexpr (P == 8) {
+        return __fadd_rn(__fadd_rn(__fadd_rn(t[0], t[1]), __fadd_rn(t[2], t[3])),
+                         __fadd_rn(__fadd_rn(t[4], t[5]), __fadd_rn(t[6], t[7])));
+    } else {
+        return t[0];
+    }
+}
+
+template <int P, bool TOPK> struct SweepAcc {
+    double s1 = 0.0, s2 = 0.0, sa = 0.0;
+    uint32_t amax = 0u, amin = 0xFFFFFFFFu, gmax = 0u, hmax = 0u;
+
+    // one element: gradient value gv, probe products hv[p], sign words sel[p], bit position pos
+    __device__ __forceinline__ uint32_t element(float gv, const float (&hv)[P > 0 ? P : 1],
+                                                const uint32_t (&sel)[P > 0 ? P : 1], uint32_t pos)
+    {
+        const uint32_t gb = __float_as_uint(gv) & 0x7FFFFFFFu;
+        gmax = max(gmax, gb);
+        const double x = (double)gv;
+        s1 += x;
+        s2 = fma(x, x, s2);
+        uint32_t ab = 0u;
+        if (P == 1) {
+            ab = __float_as_uint(hv[0]) & 0x7FFFFFFFu;       // |z h| = |h|
+        } else if (P > 1) {
+            float t[P > 0 ? P : 1];
+#pragma unroll
+            for (int p = 0; p < P; ++p) {
+                const uint32_t hb = __float_as_uint(hv[p]);
+                hmax = max(hmax, hb & 0x7FFFFFFFu);
+                t[p] = __uint_as_float(hb ^ (((sel[p] >> pos) & 1u) << 31));
+            }
+            ab = __float_as_uint(pairwise<P>(t)) & 0x7FFFFFFFu;
+        }
+        if (P > 0) {
+            amax = max(amax, ab);
+            amin = min(amin, ab);
+            if (TOPK) sa += (double)__uint_as_float(ab);
+        }
+        return ab;
+    }
+};
+
+template <int P, bool BF16, bool TOPK>
+__global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
+{
+    constexpr int PP = P > 0 ? P : 1;
+    constexpr int U = (P <= 1) ? 8 : (P == 2 ? 4 : 2);     // rows in flight per lane
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+        const uint32_t it = batch * kWarps + warp;
+        if (it >= A.n_items) continue;
+        const Item item = A.items[it];
+        const uint64_t begin = item.begin, end = begin + item.len;
+        const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
+        SweepAcc<P, TOPK> acc;
+        uint32_t X[PP][4];
+        uint64_t have_block = ~0ull;
+
+        auto refresh = [&](uint64_t row) {
+            if (P > 1) {
+                const uint64_t blk = row >> 5;
+                if (blk != have_block) {
+#pragma unroll
+                    for (int p = 0; p < PP; ++p) probe_bits(blk, lane, A.seed, A.step, (uint32_t)p, X[p]);
+                    have_block = blk;
+                }
+            }
+        };
+
+        // scalar path for a row that is not entirely inside [begin, end)
+        auto partial_row = [&](uint64_t row) {
+            refresh(row);
+            const uint32_t k = (uint32_t)(row & 31u);
+            uint32_t sel[PP];
+#pragma unroll
+            for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
+            const uint64_t i0 = row * 128ull + lane * 4u;
+#pragma unroll
+            for (uint32_t e = 0; e < 4; ++e) {
+                const uint64_t i = i0 + e;
+                if (i >= begin && i < end) {
+                    float hv[PP];
+#pragma unroll
+                    for (int p = 0; p < PP; ++p) hv[p] = (P > 0) ? __ldcs(A.hz + (uint64_t)p * A.n_total + i) : 0.f;
+                    const uint32_t ab = acc.element(GradVec<BF16>::load1(A.g, i), hv, sel, (k & 7u) * 4u + e);
+                    if (TOPK) {
+                        A.abs_s[i] = __uint_as_float(ab);
+                        atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
+                    }
+                }
+            }
+        };
+
+        auto full_rows = [&](uint64_t row, RowData<P> (&rd)[U], int count) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (u < count) {
+                    const uint32_t k = (uint32_t)((row + u) & 31u);
+                    uint32_t sel[PP];
+#pragma unroll
+                    for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
+                    const float gv[4] = {rd[u].g.x, rd[u].g.y, rd[u].g.z, rd[u].g.w};
+                    float av[4];
+#pragma unroll
+                    for (uint32_t e = 0; e < 4; ++e) {
+                        float hv[PP];
+#pragma unroll
+                        for (int p = 0; p < PP; ++p) {
+                            const float4 h = rd[u].hz[p];
+                            hv[p] = e == 0 ? h.x : (e == 1 ? h.y : (e == 2 ? h.z : h.w));
+                        }
+                        const uint32_t ab = acc.element(gv[e], hv, sel, (k & 7u) * 4u + e);
+                        av[e] = __uint_as_float(ab);
+                        if (TOPK) atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
+                    }
+                    if (TOPK) {
+                        const uint64_t i0 = (row + u) * 128ull + lane * 4u;
+                        *reinterpret_cast<float4 *>(A.abs_s + i0) = make_float4(av[0], av[1], av[2], av[3]);
+                    }
+                }
+            }
+        };
+
+        auto load_rows = [&](uint64_t row, RowData<P> (&rd)[U], int count) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (u < count) {
+                    const uint64_t i0 = (row + u) * 128ull + lane * 4u;
+                    rd[u].g = GradVec<BF16>::load4(A.g, i0, false);
+#pragma unroll
+                    for (int p = 0; p < PP; ++p)
+                        if (P > 0) rd[u].hz[p] = ld_stream(A.hz + (uint64_t)p * A.n_total + i0);
+                }
+            }
+        };
+
+        // rows [full_lo, full_hi) lie entirely inside the item; at most one partial row at each end
+        const uint64_t full_lo = (begin + 127) >> 7, full_hi = end >> 7;
+        const bool head_partial = (begin & 127u) != 0u;
+        const bool tail_partial = (end & 127u) != 0u && !(head_partial && row_last == row_first);
+        if (head_partial) partial_row(row_first);
+        if (full_hi > full_lo) {
+            uint64_t row = full_lo;
+            RowData<P> rd[U];
+            // single rows up to the next multiple of U, so that an unrolled group never crosses a 32-row block
+            while (row < full_hi && (row & (U - 1))) {
+                refresh(row);
+                load_rows(row, rd, 1);
+                full_rows(row, rd, 1);
+                ++row;
+            }
+            while (row + U <= full_hi) {
+                refresh(row);
+                load_rows(row, rd, U);
+                full_rows(row, rd, U);
+                row += U;
+            }
+            while (row < full_hi) {
+                refresh(row);
+                load_rows(row, rd, 1);
+                full_rows(row, rd, 1);
+                ++row;
+            }
+        }
+        if (tail_partial) partial_row(row_last);
+
+        // warp reduction
+        const double s1 = warp_sum(acc.s1), s2 = warp_sum(acc.s2);
+        const double sa = TOPK ? warp_sum(acc.sa) : 0.0;
+        const uint32_t amax = __reduce_max_sync(0xFFFFFFFFu, acc.amax);
+        const uint32_t amin = __reduce_min_sync(0xFFFFFFFFu, acc.amin);
+        const uint32_t gmax = __reduce_max_sync(0xFFFFFFFFu, acc.gmax);
+        const uint32_t hmax = __reduce_max_sync(0xFFFFFFFFu, P == 1 ? acc.amax : acc.hmax);
+        uint32_t bad = 0;
+        if (gmax >= kNonFiniteBits || (P > 0 && hmax >= kNonFiniteBits)) {
+            // rare: count the non-finite inputs of this item exactly
+            for (uint64_t i = begin + lane; i < end; i += 32) {
+                if ((__float_as_uint(GradVec<BF16>::load1(A.g, i)) & 0x7FFFFFFFu) >= kNonFiniteBits) ++bad;
+                for (int p = 0; p < P; ++p)
+                    if ((__float_as_uint(A.hz[(uint64_t)p * A.n_total + i]) & 0x7FFFFFFFu) >= kNonFiniteBits) ++bad;
+            }
+            bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+        }
+        if (lane == 0) {
+            A.p_s1[it] = s1;
+            A.p_s2[it] = s2;
+            A.p_bad[it] = bad;
+            if (P > 0) { A.p_amax[it] = amax; A.p_amin[it] = amin; }
+            if (TOPK) A.p_sa[it] = sa;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ decisions
+
+struct DecideArgs {
+    const uint32_t *item_lo;        // [L + 1] first item of each layer
+    const uint64_t *seg_len;        // [L]
+    const double *p_s1, *p_s2, *p_sa;
+    const uint32_t *p_amax, *p_amin, *p_bad;
+    LayerScratch *scratch;          // [L]
+    LayerState *state;              // [L]
+    Status *status;
+    Hyper hp;
+    float eta0;
+    uint32_t L;
+    uint32_t has_hz, control, topk;
+    unsigned long long step;
+};
+
+// Reads another block's results past the L1 cache (they were published with a fence).
+__device__ __forceinline__ LayerScratch load_scratch(const LayerScratch *p)
+{
+    LayerScratch sc;
+    sc.mean = __ldcg(&p->mean);
+    sc.var = __ldcg(&p->var);
+    sc.sum_abs = __ldcg(&p->sum_abs);
+    sc.bad = __ldcg(&p->bad);
+    sc.amax = __ldcg(&p->amax);
+    sc.amin = __ldcg(&p->amin);
+    return sc;
+}
+
+// Sec. 3.1 (EMAs, code cases), Sec. 3.2 (step size, promotion), Sec. 3.4 (control interval).
+__device__ __forceinline__ uint32_t commit_layer(const DecideArgs &A, uint32_t l)
+{
+    LayerState st = A.state[l];
+    const LayerScratch sc = load_scratch(A.scratch + l);
+    const double beta = (double)A.hp.beta;
+    st.grad_mean = sc.mean;
+    st.grad_var = sc.var;
+    st.ema_mean = (float)(beta * (double)st.ema_mean + (1.0 - beta) * sc.mean);
+    st.ema_var = (float)(beta * (double)st.ema_var + (1.0 - beta) * sc.var);
+    if (A.has_hz) {
+        st.lambda_max = __fdiv_rn(__uint_as_float(sc.amax), (float)A.hp.num_probes);
+        if (!A.topk) { st.thr = __uint_as_float(sc.amin); st.topk_mass = 1.0; }
+    }
+    uint32_t near = 0;
+    if (A.control) {
+        const float v = st.ema_var;
+        uint32_t code = v < A.hp.tau_low ? 0u : (v < A.hp.tau_high ? 1u : 2u);
+        if (st.lambda_max > A.hp.tau_curv && code < 2u) code += 1u;
+        st.code = code;
+        st.eta_scale = __fdiv_rn(1.0f, __fadd_rn(1.0f, __fmul_rn(A.hp.alpha, st.lambda_max)));
+        if (fabs((double)v - (double)A.hp.tau_low) <= 1e-5 * fabs((double)A.hp.tau_low)) near = 1;
+        if (fabs((double)v - (double)A.hp.tau_high) <= 1e-5 * fabs((double)A.hp.tau_high)) near = 1;
+        if (fabs((double)st.lambda_max - (double)A.hp.tau_curv) <= 1e-5 * fabs((double)A.hp.tau_curv)) near = 1;
+        st.near = near;
+    }
+    st.eta = __fmul_rn(A.eta0, st.eta_scale);
+    A.state[l] = st;
+    return near;
+}
+
+// One block per layer combines the layer's item partials in a fixed order; the block that
+// finishes last screens the whole step for non-finite input and commits every layer.
+__global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
+{
+    __shared__ double red[kWarps];
+    __shared__ uint32_t red_u[2][kWarps];
+    __shared__ uint32_t is_last;
+    const uint32_t l = blockIdx.x, tid = threadIdx.x;
+    const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
+    double s1 = 0.0, s2 = 0.0, sa = 0.0, bad = 0.0;
+    uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+    for (uint32_t i = lo + tid; i < hi; i += kThreads) {
+        s1 += A.p_s1[i];
+        s2 += A.p_s2[i];
+        bad += (double)A.p_bad[i];
+        if (A.has_hz) {
+            amax = max(amax, A.p_amax[i]);
+            amin = min(amin, A.p_amin[i]);
+            if (A.topk) sa += A.p_sa[i];
+        }
+    }
+    s1 = block_sum(s1, red);
+    s2 = block_sum(s2, red);
+    sa = block_sum(sa, red);
+    bad = block_sum(bad, red);
+    amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+    amin = __reduce_min_sync(0xFFFFFFFFu, amin);
+    if ((tid & 31) == 0) { red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
+        const double n = (double)A.seg_len[l];
+        const double mu = s1 / n;
+        double var = s2 / n - mu * mu;
+        if (!(var > 0.0)) var = 0.0;
+        LayerScratch sc;
+        sc.mean = mu; sc.var = var; sc.sum_abs = sa;
+        sc.bad = (unsigned long long)bad;
+        sc.amax = amax; sc.amin = amin;
+        A.scratch[l] = sc;
+        __threadfence();
+        const uint32_t ticket = atomicAdd(&A.status->done_counter, 1u);
+        is_last = (ticket == A.L - 1) ? 1u : 0u;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double total_bad = 0.0;
+    for (uint32_t j = tid; j < A.L; j += kThreads)
+        total_bad += (double)__ldcg(&A.scratch[j].bad);
+    total_bad = block_sum(total_bad, red);
+    double near = 0.0;
+    if (total_bad == 0.0)
+        for (uint32_t j = tid; j < A.L; j += kThreads) near += (double)commit_layer(A, j);
+    near = block_sum(near, red);
+    if (tid == 0) {
+        A.status->step = A.step;
+        A.status->nonfinite = (unsigned long long)total_bad;
+        A.status->skipped = total_bad != 0.0 ? 1u : 0u;
+        if (A.control && total_bad == 0.0) A.status->near_count = (uint32_t)near;
+        A.status->done_counter = 0u;
+    }
+}
+
+// ------------------------------------------------------------------ phase B: update + cast
+
+struct ApplyArgs {
+    const Item *items;
+    uint32_t n_items, n_batches;
+    float *w;
+    const void *g;
+    uint16_t *c;
+    const LayerState *state;
+    const Status *status;
+};
+
+__device__ __forceinline__ uint16_t cast16(float x, uint32_t code)
+{
+    return code == 0u ? __half_as_ushort(__float2half_rn(x)) : __bfloat16_as_ushort(__float2bfloat16_rn(x));
+}
+
+// w <- fl32(w - eta_l g) (Sec. 3.2, Sec. 4.1); c <- RNE cast of the new w for FP16 / BF16 layers (Sec. 2).
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
+{
+    if (A.status->skipped) return;
+    constexpr int U = 4;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+        const uint32_t it = batch * kWarps + warp;
+        if (it >= A.n_items) continue;
+        const Item item = A.items[it];
+        const uint64_t begin = item.begin, end = begin + item.len;
+        const float neg_eta = -A.state[item.seg].eta;
+        const uint32_t code = A.state[item.seg].code;
+
+        auto partial_row = [&](uint64_t row) {
+            const uint64_t i0 = row * 128ull + lane * 4u;
+            for (uint32_t e = 0; e < 4; ++e) {
+                const uint64_t i = i0 + e;
+                if (i >= begin && i < end) {
+                    const float wn = fmaf(neg_eta, GradVec<BF16>::load1(A.g, i), A.w[i]);
+                    A.w[i] = wn;
+                    if (code < 2u) A.c[i] = cast16(wn, code);
+                }
+            }
+        };
+        auto store_row = [&](uint64_t i0, float4 wv, float4 gv) {
+            wv.x = fmaf(neg_eta, gv.x, wv.x);
+            wv.y = fmaf(neg_eta, gv.y, wv.y);
+            wv.z = fmaf(neg_eta, gv.z, wv.z);
+            wv.w = fmaf(neg_eta, gv.w, wv.w);
+            *reinterpret_cast<float4 *>(A.w + i0) = wv;
+            if (code == 0u) {
+                const __half2 a = __floats2half2_rn(wv.x, wv.y), b = __floats2half2_rn(wv.z, wv.w);
+                uint2 o;
+                o.x = *reinterpret_cast<const uint32_t *>(&a);
+                o.y = *reinterpret_cast<const uint32_t *>(&b);
+                __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
+            } else if (code == 1u) {
+                const __nv_bfloat162 a = __floats2bfloat162_rn(wv.x, wv.y), b = __floats2bfloat162_rn(wv.z, wv.w);
+                uint2 o;
+                o.x = *reinterpret_cast<const uint32_t *>(&a);
+                o.y = *reinterpret_cast<const uint32_t *>(&b);
+                __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
+            }
+        };
+
+        const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
+        const uint64_t full_lo = (begin + 127) >> 7, full_hi = end >> 7;
+        const bool head_partial = (begin & 127u) != 0u;
+        const bool tail_partial = (end & 127u) != 0u && !(head_partial && row_last == row_first);
+        if (head_partial) partial_row(row_first);
+        if (full_hi > full_lo) {
+            uint64_t row = full_lo;
+            while (row + U <= full_hi) {
+                float4 wv[U], gv[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint64_t i0 = (row + u) * 128ull + lane * 4u;
+                    wv[u] = ld_stream(A.w + i0);
+                    gv[u] = GradVec<BF16>::load4(A.g, i0, true);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) store_row((row + u) * 128ull + lane * 4u, wv[u], gv[u]);
+                row += U;
+            }
+            while (row < full_hi) {
+                const uint64_t i0 = row * 128ull + lane * 4u;
+                store_row(i0, ld_stream(A.w + i0), GradVec<BF16>::load4(A.g, i0, true));
+                ++row;
+            }
+        }
+        if (tail_partial) partial_row(row_last);
+    }
+}
+
+// ------------------------------------------------------------------ probe writer
+
+__global__ void __launch_bounds__(kThreads) k_probe(float *z, uint64_t n_vec, uint64_t seed, uint32_t step, uint32_t p)
+{
+    for (uint64_t v = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; v < n_vec; v += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t i0 = v * 4ull;
+        const uint64_t row = i0 >> 7;
+        const uint32_t k = (uint32_t)(row & 31u), slot = (uint32_t)(v & 31u);
+        uint32_t x[4];
+        probe_bits(row >> 5, slot, seed, step, p, x);
+        const uint32_t bits = pick_word(x, k >> 3) >> ((k & 7u) * 4u);
+        float4 o;
+        o.x = (bits & 1u) ? -1.f : 1.f;
+        o.y = (bits & 2u) ? -1.f : 1.f;
+        o.z = (bits & 4u) ? -1.f : 1.f;
+        o.w = (bits & 8u) ? -1.f : 1.f;
+        *reinterpret_cast<float4 *>(z + i0) = o;
+    }
+}
+
+// ------------------------------------------------------------------ top-k: radix select on |S| bit patterns
+
+struct SelectArgs {
+    uint32_t *hist;              // [L][kHistBins]
+    SelectState *sel;            // [L]
+    LayerState *state;           // [L]
+    const uint64_t *seg_k;       // [L] mask population
+    const Status *status;
+};
+
+// LEVEL 1: bits 30..20, LEVEL 2: bits 19..9, LEVEL 3: bits 8..0.  One block per layer: finds the
+// bin in which the k-th largest element falls and how many elements are still to be taken in it.
+template <int LEVEL>
+__global__ void __launch_bounds__(kThreads) k_select(const SelectArgs A)
+{
+    constexpr int BINS = LEVEL == 3 ? 512 : kHistBins;
+    constexpr int PER = BINS / kThreads;            // bins per thread, taken from the top down
+    __shared__ uint32_t h[BINS];
+    __shared__ uint32_t chunk[kThreads];
+    const uint32_t l = blockIdx.x, tid = threadIdx.x;
+    uint32_t *gh = A.hist + (uint64_t)l * kHistBins;
+    for (int b = tid; b < BINS; b += kThreads) { h[b] = gh[b]; gh[b] = 0u; }
+    if (A.status->skipped) return;
+    __syncthreads();
+    // thread t owns bins BINS-1-PER*t .. BINS-PER*(t+1), in descending order
+    uint32_t mine = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) mine += h[BINS - 1 - (PER * (int)tid + j)];
+    chunk[tid] = mine;
+    __syncthreads();
+    // inclusive scan over threads (Hillis-Steele)
+    for (int o = 1; o < kThreads; o <<= 1) {
+        const uint32_t add = tid >= (uint32_t)o ? chunk[tid - o] : 0u;
+        __syncthreads();
+        chunk[tid] += add;
+        __syncthreads();
+    }
+    const uint32_t need = LEVEL == 1 ? (uint32_t)A.seg_k[l] : A.sel[l].remaining;
+    const uint32_t above = chunk[tid] - mine;       // elements in bins above this thread's bins
+    if (above < need && need <= chunk[tid]) {
+        uint32_t cum = above;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int b = BINS - 1 - (PER * (int)tid + j);
+            const uint32_t cnt = h[b];
+            if (cum < need && need <= cum + cnt) {
+                SelectState s = A.sel[l];
+                s.prefix = LEVEL == 1 ? (uint32_t)b : ((s.prefix << (LEVEL == 3 ? 9 : 11)) | (uint32_t)b);
+                s.remaining = need - cum;
+                if (LEVEL == 3) {
+                    s.thr_bits = s.prefix;
+                    s.take_equal = s.remaining;
+                    s.surplus = cnt > s.remaining ? 1u : 0u;
+                    A.state[l].thr = __uint_as_float(s.thr_bits);
+                }
+                A.sel[l] = s;
+            }
+            cum += cnt;
+        }
+    }
+}
+
+struct RefineArgs {
+    const Item *items;
+    uint32_t n_items, n_batches;
+    const float *abs_s;
+    uint32_t *hist;
+    const SelectState *sel;
+    const Status *status;
+};
+
+// Histogram of the next digit over the elements whose higher bits equal the layer's prefix.
+template <int LEVEL>
+__global__ void __launch_bounds__(kThreads) k_refine(const RefineArgs A)
+{
+    if (A.status->skipped) return;
+    constexpr int SHIFT_PREFIX = LEVEL == 2 ? 20 : 9;
+    constexpr int SHIFT_DIGIT = LEVEL == 2 ? 9 : 0;
+    constexpr uint32_t DIGIT_MASK = LEVEL == 2 ? 2047u : 511u;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+        const uint32_t it = batch * kWarps + warp;
+        if (it >= A.n_items) continue;
+        const Item item = A.items[it];
+        const uint64_t begin = item.begin, end = begin + item.len;
+        const uint32_t prefix = A.sel[item.seg].prefix;
+        uint32_t *hist = A.hist + (uint64_t)item.seg * kHistBins;
+        const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
+        for (uint64_t row = row_first; row <= row_last; ++row) {
+            const uint64_t i0 = row * 128ull + lane * 4u;
+            const bool full = row * 128ull >= begin && row * 128ull + 128u <= end;
+            uint32_t ab[4];
+            bool ok[4];
+            if (full) {
+                const float4 v = __ldg(reinterpret_cast<const float4 *>(A.abs_s + i0));
+                ab[0] = __float_as_uint(v.x); ab[1] = __float_as_uint(v.y);
+                ab[2] = __float_as_uint(v.z); ab[3] = __float_as_uint(v.w);
+                ok[0] = ok[1] = ok[2] = ok[3] = true;
+            } else {
+                for (uint32_t e = 0; e < 4; ++e) {
+                    ok[e] = i0 + e >= begin && i0 + e < end;
+                    ab[e] = ok[e] ? __float_as_uint(A.abs_s[i0 + e]) : 0u;
+                }
+            }
+#pragma unroll
+            for (uint32_t e = 0; e < 4; ++e) {
+                const bool hit = ok[e] && (ab[e] >> SHIFT_PREFIX) == prefix;
+                const uint32_t digit = (ab[e] >> SHIFT_DIGIT) & DIGIT_MASK;
+                // the whole warp is converged here: aggregate the common case of one shared digit
+                const uint32_t m = __ballot_sync(0xFFFFFFFFu, hit);
+                if (m) {
+                    const int leader = __ffs(m) - 1;
+                    const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, leader);
+                    const uint32_t same = __ballot_sync(0xFFFFFFFFu, hit && digit == d0);
+                    if (same == m) {
+                        if ((int)lane == leader) atomicAdd(hist + d0, (uint32_t)__popc(m));
+                    } else if (hit) {
+                        atomicAdd(hist + digit, 1u);
+                    }
+                }
+            }
+        }
+    }
+}
+
+struct MaskArgs {
+    const Item *items;
+    uint32_t n_items, n_batches;
+    const float *abs_s;
+    uint32_t *mask;
+    double *p_mass;              // per item: sum of |S| strictly above the threshold
+    const SelectState *sel;
+    const Status *status;
+};
+
+__global__ void __launch_bounds__(kThreads) k_zero_mask(uint32_t *mask, uint64_t words, const Status *status)
+{
+    if (status->skipped) return;
+    for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < words; i += (uint64_t)gridDim.x * blockDim.x)
+        mask[i] = 0u;
+}
+
+// Sets the bit of every element above the threshold, and of those equal to it when all of them
+// belong to the mask; a layer with surplus ties gets its equal elements from k_finish.
+__global__ void __launch_bounds__(kThreads) k_mask(const MaskArgs A)
+{
+    if (A.status->skipped) return;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+        const uint32_t it = batch * kWarps + warp;
+        if (it >= A.n_items) continue;
+        const Item item = A.items[it];
+        const uint64_t begin = item.begin, end = begin + item.len;
+        const SelectState s = A.sel[item.seg];
+        const uint32_t ge = s.surplus ? s.thr_bits + 1u : s.thr_bits;   // take bit patterns >= ge
+        double mass = 0.0;
+        const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
+        for (uint64_t row = row_first; row <= row_last; ++row) {
+            const uint64_t i0 = row * 128ull + lane * 4u;
+            const bool full = row * 128ull >= begin && row * 128ull + 128u <= end;
+            uint32_t nib = 0u;
+            if (full) {
+                const float4 v = __ldcs(reinterpret_cast<const float4 *>(A.abs_s + i0));
+                const float av[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (uint32_t e = 0; e < 4; ++e) {
+                    const uint32_t ab = __float_as_uint(av[e]);
+                    if (ab >= ge) nib |= 1u << e;
+                    if (ab > s.thr_bits) mass += (double)av[e];
+                }
+            } else {
+                for (uint32_t e = 0; e < 4; ++e) {
+                    if (i0 + e >= begin && i0 + e < end) {
+                        const float a = A.abs_s[i0 + e];
+                        const uint32_t ab = __float_as_uint(a);
+                        if (ab >= ge) nib |= 1u << e;
+                        if (ab > s.thr_bits) mass += (double)a;
+                    }
+                }
+            }
+            uint32_t word = nib << ((lane & 7u) * 4u);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+            if ((lane & 7u) == 0u) {
+                uint32_t *dst = A.mask + (row * 4ull + (lane >> 3));
+                if (full) *dst = word;
+                else if (word) atomicOr(dst, word);
+            }
+        }
+        mass = warp_sum(mass);
+        if (lane == 0) A.p_mass[it] = mass;
+    }
+}
+
+struct FinishArgs {
+    const uint32_t *item_lo;
+    const ta::Item *items;
+    const uint64_t *seg_off, *seg_len;
+    const float *abs_s;
+    uint32_t *mask;
+    const double *p_mass;
+    const LayerScratch *scratch;
+    const SelectState *sel;
+    LayerState *state;
+    const Status *status;
+};
+
+// One block per layer: the masked share of |S|, and, for a layer with surplus ties at the
+// threshold, the bits of the first take_equal elements equal to it, in index order.
+__global__ void __launch_bounds__(kThreads) k_finish(const FinishArgs A)
+{
+    if (A.status->skipped) return;
+    __shared__ double red[kWarps];
+    __shared__ uint32_t wsum[kWarps];
+    const uint32_t l = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const SelectState s = A.sel[l];
+    double mass = 0.0;
+    for (uint32_t i = A.item_lo[l] + tid; i < A.item_lo[l + 1]; i += kThreads) mass += A.p_mass[i];
+    mass = block_sum(mass, red);
+    if (tid == 0) {
+        const double all = A.scratch[l].sum_abs;
+        const double masked = mass + (double)s.take_equal * (double)__uint_as_float(s.thr_bits);
+        A.state[l].topk_mass = all > 0.0 ? masked / all : 1.0;
+    }
+    if (!s.surplus) return;
+    const uint64_t off = A.seg_off[l], n = A.seg_len[l];
+    uint32_t taken = 0;
+    for (uint64_t base = 0; base < n && taken < s.take_equal; base += kThreads) {
+        const uint64_t j = base + tid;
+        const bool eq = j < n && __float_as_uint(A.abs_s[off + j]) == s.thr_bits;
+        const uint32_t m = __ballot_sync(0xFFFFFFFFu, eq);
+        __syncthreads();
+        if (lane == 0) wsum[warp] = (uint32_t)__popc(m);
+        __syncthreads();
+        uint32_t before = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            if (w < (int)warp) before += wsum[w];
+            total += wsum[w];
+        }
+        const uint32_t rank = taken + before + (uint32_t)__popc(m & ((1u << lane) - 1u));
+        if (eq && rank < s.take_equal) {
+            const uint64_t i = off + j;
+            atomicOr(A.mask + (i >> 5), 1u << (i & 31u));
+        }
+        taken += total;
+    }
+}
+
+}  // namespace ta

@@ -1,0 +1,619 @@
+// Host side of the Tri-Accel optimizer pass: C ABI, planner, launches.  See include/triaccel.h
+// for the contract of every entry point.
+#include "../../include/triaccel.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kernels.cuh"
+
+namespace {
+
+thread_local char g_create_error[256] = "";
+
+struct DeviceBuffers {
+    ta::Item *items = nullptr;
+    uint32_t *item_lo = nullptr;
+    uint64_t *seg_off = nullptr, *seg_len = nullptr, *seg_k = nullptr;
+    ta::LayerState *state = nullptr;
+    ta::LayerScratch *scratch = nullptr;
+    ta::Status *status = nullptr;
+    double *p_s1 = nullptr, *p_s2 = nullptr, *p_sa = nullptr, *p_mass = nullptr;
+    uint32_t *p_amax = nullptr, *p_amin = nullptr, *p_bad = nullptr;
+    float *abs_s = nullptr;
+    uint32_t *hist = nullptr;
+    ta::SelectState *sel = nullptr;
+    uint32_t *mask = nullptr;
+    // host-tensor staging (ta_step_host)
+    float *st_w = nullptr, *st_hz = nullptr;
+    void *st_g = nullptr;
+    uint16_t *st_c = nullptr;
+};
+
+}  // namespace
+
+struct ta_handle {
+    int device = 0;
+    int sm_count = 0;
+    uint32_t L = 0;
+    uint64_t n_total = 0;
+    ta_hparams hp{};
+    std::vector<ta_segment> table;
+    std::vector<uint64_t> seg_k;
+    uint32_t n_items = 0, n_batches = 0, item_elems = 0;
+    uint64_t mask_words = 0;
+    bool topk = false;
+    bool stepped = false;
+    uint64_t last_step = 0;
+    uint64_t launches = 0;
+    cudaStream_t last_stream = nullptr;
+    std::vector<cudaEvent_t> events;      // 4 per timed step: before sweep, after sweep, after decisions, after update
+    uint32_t timed_cap = 0, timed_used = 0;
+    DeviceBuffers d;
+    char err[256] = "";
+};
+
+namespace {
+
+int fail(ta_handle *h, int code, const char *fmt, const char *detail = "")
+{
+    char *dst = h ? h->err : g_create_error;
+    snprintf(dst, 256, fmt, detail);
+    return code;
+}
+
+#define TA_CUDA(h, call)                                                          \
+    do {                                                                          \
+        cudaError_t e__ = (call);                                                 \
+        if (e__ != cudaSuccess) {                                                 \
+            char *dst__ = (h) ? (h)->err : g_create_error;                        \
+            snprintf(dst__, 256, "%s failed: %s", #call, cudaGetErrorString(e__)); \
+            return e__ == cudaErrorMemoryAllocation ? TA_ERR_NOMEM : TA_ERR_CUDA; \
+        }                                                                         \
+    } while (0)
+
+template <typename T> cudaError_t dev_alloc(T **p, size_t count)
+{
+    return cudaMalloc(reinterpret_cast<void **>(p), std::max<size_t>(count, 1) * sizeof(T));
+}
+
+void free_all(DeviceBuffers &d)
+{
+    void *ptrs[] = {d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
+                    d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.st_w, d.st_hz,
+                    d.st_g, d.st_c};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+    d = DeviceBuffers{};
+}
+
+// Elements per work item: the largest size that still gives every warp slot of the GPU a few
+// items, so that thousands of tiny tensors and a few huge ones both keep all SMs busy.
+uint32_t choose_item_elems(uint64_t n_params, int sm_count)
+{
+    if (const char *env = getenv("TRIACCEL_ITEM_ELEMS")) {
+        const long v = atol(env);
+        if (v >= 128 && v <= (1 << 20) && v % 128 == 0) return (uint32_t)v;
+    }
+    const uint64_t want_items = (uint64_t)sm_count * ta::kWarps * 4;
+    uint32_t best = 512;
+    for (uint32_t cand : {1024u, 2048u, 4096u, 8192u, 16384u})
+        if (n_params / cand >= want_items) best = cand;
+    return best;
+}
+
+int grid_for(const ta_handle *h)
+{
+    int per_sm = 8;
+    if (const char *env = getenv("TRIACCEL_CTAS_PER_SM")) {
+        const int v = atoi(env);
+        if (v >= 1 && v <= 32) per_sm = v;
+    }
+    const long long cap = (long long)h->sm_count * per_sm;
+    return (int)std::max<long long>(1, std::min<long long>(h->n_batches, cap));
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+ta::Hyper hyper_of(const ta_hparams &hp)
+{
+    ta::Hyper y;
+    y.beta = hp.beta; y.tau_low = hp.tau_low; y.tau_high = hp.tau_high; y.tau_curv = hp.tau_curv;
+    y.alpha = hp.alpha; y.num_probes = hp.num_probes; y.t_ctrl = hp.t_ctrl; y.topk_ppm = hp.topk_ppm;
+    return y;
+}
+
+template <int P, bool BF16, bool TOPK> void launch_sweep(ta_handle *h, const ta::SweepArgs &a, cudaStream_t s)
+{
+    ta::k_sweep<P, BF16, TOPK><<<grid_for(h), ta::kThreads, 0, s>>>(a);
+    ++h->launches;
+}
+
+template <bool BF16> bool dispatch_sweep(ta_handle *h, int P, const ta::SweepArgs &a, cudaStream_t s)
+{
+    const bool topk = h->topk && P > 0;
+    switch (P) {
+    case 0: launch_sweep<0, BF16, false>(h, a, s); return true;
+    case 1: topk ? launch_sweep<1, BF16, true>(h, a, s) : launch_sweep<1, BF16, false>(h, a, s); return true;
+    case 2: topk ? launch_sweep<2, BF16, true>(h, a, s) : launch_sweep<2, BF16, false>(h, a, s); return true;
+    case 4: topk ? launch_sweep<4, BF16, true>(h, a, s) : launch_sweep<4, BF16, false>(h, a, s); return true;
+    case 8: topk ? launch_sweep<8, BF16, true>(h, a, s) : launch_sweep<8, BF16, false>(h, a, s); return true;
+    default: return false;
+    }
+}
+
+int default_mem_reader(void *, uint64_t *free_b, uint64_t *total_b)
+{
+    size_t f = 0, t = 0;
+    if (cudaMemGetInfo(&f, &t) != cudaSuccess) return 1;
+    *free_b = f;
+    *total_b = t;
+    return 0;
+}
+
+struct StateHeader {
+    uint64_t magic, n_total, last_step, mask_words;
+    uint32_t L, stepped;
+    ta_hparams hp;
+};
+constexpr uint64_t kStateMagic = 0x5441535441544531ull;   // "TASTATE1"
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+const char *ta_last_error(const ta_handle *h) { return h ? h->err : g_create_error; }
+
+int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hparams *hp, ta_handle **out)
+{
+    if (out) *out = nullptr;
+    g_create_error[0] = 0;
+    if (!table || !hp || !out || L == 0) return fail(nullptr, TA_ERR_ARG, "ta_create: NULL argument or empty table");
+    if (hp->struct_size != sizeof(ta_hparams)) return fail(nullptr, TA_ERR_ARG, "ta_create: hp.struct_size does not match this library");
+    if (!(hp->beta >= 0.f && hp->beta < 1.f)) return fail(nullptr, TA_ERR_ARG, "ta_create: beta must be in [0,1)");
+    if (!(hp->tau_low <= hp->tau_high)) return fail(nullptr, TA_ERR_ARG, "ta_create: tau_low must not exceed tau_high");
+    if (!(hp->alpha >= 0.f)) return fail(nullptr, TA_ERR_ARG, "ta_create: alpha must be >= 0");
+    if (hp->num_probes != 1 && hp->num_probes != 2 && hp->num_probes != 4 && hp->num_probes != 8)
+        return fail(nullptr, TA_ERR_ARG, "ta_create: num_probes must be 1, 2, 4 or 8");
+    if (hp->topk_ppm == 0 || hp->topk_ppm > 1000000u) return fail(nullptr, TA_ERR_ARG, "ta_create: topk_ppm must be in [1, 1000000]");
+    if (hp->t_ctrl == 0) return fail(nullptr, TA_ERR_ARG, "ta_create: t_ctrl must be >= 1");
+    if (hp->grad_dtype != TA_GRAD_F32 && hp->grad_dtype != TA_GRAD_BF16) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown grad_dtype");
+    if (hp->momentum != 0.f || hp->weight_decay != 0.f || hp->flags != 0u)
+        return fail(nullptr, TA_ERR_ARG, "ta_create: momentum, weight_decay and flags must be 0");
+    if (n_total % 4 != 0) return fail(nullptr, TA_ERR_ARG, "ta_create: n_total must be a multiple of 4");
+    uint64_t end = 0, n_params = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        if (table[l].length == 0 || table[l].length > 0xFFFFFFFEull)
+            return fail(nullptr, TA_ERR_ARG, "ta_create: segment length out of range");
+        if (table[l].offset < end) return fail(nullptr, TA_ERR_ARG, "ta_create: segments must be ascending and non-overlapping");
+        end = table[l].offset + table[l].length;
+        n_params += table[l].length;
+    }
+    if (end > n_total) return fail(nullptr, TA_ERR_ARG, "ta_create: a segment reaches beyond n_total");
+
+    ta_handle *h = new (std::nothrow) ta_handle;
+    if (!h) return fail(nullptr, TA_ERR_NOMEM, "ta_create: out of host memory");
+    auto bail = [&](int code) {
+        snprintf(g_create_error, 256, "%s", h->err);
+        free_all(h->d);
+        delete h;
+        return code;
+    };
+#define TA_TRY(call)                                                                 \
+    do {                                                                             \
+        cudaError_t e__ = (call);                                                    \
+        if (e__ != cudaSuccess) {                                                    \
+            snprintf(h->err, 256, "%s failed: %s", #call, cudaGetErrorString(e__));  \
+            return bail(e__ == cudaErrorMemoryAllocation ? TA_ERR_NOMEM : TA_ERR_CUDA); \
+        }                                                                            \
+    } while (0)
+
+    TA_TRY(cudaGetDevice(&h->device));
+    cudaDeviceProp prop;
+    TA_TRY(cudaGetDeviceProperties(&prop, h->device));
+    if (prop.major < 10) {
+        snprintf(h->err, 256, "ta_create: device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+        return bail(TA_ERR_CUDA);
+    }
+    h->sm_count = prop.multiProcessorCount;
+    h->L = L;
+    h->n_total = n_total;
+    h->hp = *hp;
+    h->table.assign(table, table + L);
+    h->topk = hp->topk_ppm < 1000000u;
+    h->mask_words = h->topk ? (n_total + 31) / 32 : 0;
+
+    // plan: items cut on a global grid of item_elems elements, clipped to each layer
+    h->item_elems = choose_item_elems(n_params, h->sm_count);
+    std::vector<ta::Item> items;
+    std::vector<uint32_t> item_lo(L + 1);
+    std::vector<uint64_t> seg_off(L), seg_len(L);
+    h->seg_k.resize(L);
+    for (uint32_t l = 0; l < L; ++l) {
+        item_lo[l] = (uint32_t)items.size();
+        const uint64_t b = table[l].offset, e = b + table[l].length;
+        seg_off[l] = b;
+        seg_len[l] = table[l].length;
+        uint64_t k = (table[l].length * (uint64_t)hp->topk_ppm + 999999ull) / 1000000ull;
+        h->seg_k[l] = k < 1 ? 1 : k;
+        for (uint64_t p = b; p < e;) {
+            const uint64_t next = std::min(e, (p / h->item_elems + 1) * (uint64_t)h->item_elems);
+            items.push_back(ta::Item{p, (uint32_t)(next - p), l});
+            p = next;
+        }
+        if (items.size() > 0x7FFFFFFFull) { snprintf(h->err, 256, "ta_create: too many work items"); return bail(TA_ERR_ARG); }
+    }
+    item_lo[L] = (uint32_t)items.size();
+    h->n_items = (uint32_t)items.size();
+    h->n_batches = (h->n_items + ta::kWarps - 1) / ta::kWarps;
+
+    DeviceBuffers &d = h->d;
+    TA_TRY(dev_alloc(&d.items, items.size()));
+    TA_TRY(dev_alloc(&d.item_lo, L + 1));
+    TA_TRY(dev_alloc(&d.seg_off, L));
+    TA_TRY(dev_alloc(&d.seg_len, L));
+    TA_TRY(dev_alloc(&d.seg_k, L));
+    TA_TRY(dev_alloc(&d.state, L));
+    TA_TRY(dev_alloc(&d.scratch, L));
+    TA_TRY(dev_alloc(&d.status, 1));
+    TA_TRY(dev_alloc(&d.p_s1, h->n_items));
+    TA_TRY(dev_alloc(&d.p_s2, h->n_items));
+    TA_TRY(dev_alloc(&d.p_amax, h->n_items));
+    TA_TRY(dev_alloc(&d.p_amin, h->n_items));
+    TA_TRY(dev_alloc(&d.p_bad, h->n_items));
+    if (h->topk) {
+        TA_TRY(dev_alloc(&d.p_sa, h->n_items));
+        TA_TRY(dev_alloc(&d.p_mass, h->n_items));
+        TA_TRY(dev_alloc(&d.abs_s, n_total));
+        TA_TRY(dev_alloc(&d.hist, (size_t)L * ta::kHistBins));
+        TA_TRY(dev_alloc(&d.sel, L));
+        TA_TRY(dev_alloc(&d.mask, h->mask_words));
+        TA_TRY(cudaMemset(d.hist, 0, (size_t)L * ta::kHistBins * sizeof(uint32_t)));
+        TA_TRY(cudaMemset(d.sel, 0, (size_t)L * sizeof(ta::SelectState)));
+        TA_TRY(cudaMemset(d.mask, 0, h->mask_words * sizeof(uint32_t)));
+    }
+    TA_TRY(cudaMemcpy(d.items, items.data(), items.size() * sizeof(ta::Item), cudaMemcpyHostToDevice));
+    TA_TRY(cudaMemcpy(d.item_lo, item_lo.data(), (L + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    TA_TRY(cudaMemcpy(d.seg_off, seg_off.data(), L * sizeof(uint64_t), cudaMemcpyHostToDevice));
+    TA_TRY(cudaMemcpy(d.seg_len, seg_len.data(), L * sizeof(uint64_t), cudaMemcpyHostToDevice));
+    TA_TRY(cudaMemcpy(d.seg_k, h->seg_k.data(), L * sizeof(uint64_t), cudaMemcpyHostToDevice));
+    std::vector<ta::LayerState> init(L);
+    for (auto &s : init) {
+        std::memset(&s, 0, sizeof(s));
+        s.code = TA_CODE_BF16;        // BF16 is the default mode (Sec. 3.1)
+        s.eta_scale = 1.0f;
+        s.eta = hp->eta0;
+        s.topk_mass = 0.0;
+    }
+    TA_TRY(cudaMemcpy(d.state, init.data(), L * sizeof(ta::LayerState), cudaMemcpyHostToDevice));
+    TA_TRY(cudaMemset(d.scratch, 0, L * sizeof(ta::LayerScratch)));
+    TA_TRY(cudaMemset(d.status, 0, sizeof(ta::Status)));
+    TA_TRY(cudaDeviceSynchronize());
+#undef TA_TRY
+    *out = h;
+    return TA_OK;
+}
+
+int ta_destroy(ta_handle *h)
+{
+    if (!h) return TA_OK;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(h->device);
+    if (h->last_stream || h->stepped) cudaStreamSynchronize(h->last_stream);
+    for (cudaEvent_t e : h->events) cudaEventDestroy(e);
+    free_all(h->d);
+    cudaSetDevice(prev);
+    delete h;
+    return TA_OK;
+}
+
+int ta_set_lr(ta_handle *h, float eta0)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!(eta0 == eta0)) return fail(h, TA_ERR_ARG, "ta_set_lr: eta0 is NaN");
+    h->hp.eta0 = eta0;
+    return TA_OK;
+}
+
+int ta_launch_count(ta_handle *h, uint64_t *count)
+{
+    if (!h || !count) return TA_ERR_ARG;
+    *count = h->launches;
+    return TA_OK;
+}
+
+int ta_timing_begin(ta_handle *h, uint32_t max_steps)
+{
+    if (!h) return TA_ERR_ARG;
+    if (max_steps > 4096) return fail(h, TA_ERR_ARG, "ta_timing_begin: at most 4096 steps");
+    while (h->events.size() < 4 * (size_t)max_steps) {
+        cudaEvent_t e;
+        TA_CUDA(h, cudaEventCreate(&e));
+        h->events.push_back(e);
+    }
+    h->timed_cap = max_steps;
+    h->timed_used = 0;
+    return TA_OK;
+}
+
+int ta_timing_end(ta_handle *h, double *ms_sweep, double *ms_decide, double *ms_update, uint32_t *steps)
+{
+    if (!h || !ms_sweep || !ms_decide || !ms_update || !steps) return TA_ERR_ARG;
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    double acc[3] = {0.0, 0.0, 0.0};
+    for (uint32_t i = 0; i < h->timed_used; ++i)
+        for (int k = 0; k < 3; ++k) {
+            float ms = 0.f;
+            TA_CUDA(h, cudaEventElapsedTime(&ms, h->events[4 * (size_t)i + k], h->events[4 * (size_t)i + k + 1]));
+            acc[k] += ms;
+        }
+    *ms_sweep = acc[0]; *ms_decide = acc[1]; *ms_update = acc[2];
+    *steps = h->timed_used;
+    h->timed_cap = 0;
+    h->timed_used = 0;
+    return TA_OK;
+}
+
+int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c, uint64_t probe_seed, uint64_t step,
+            void *stream)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!w || !g || !c) return fail(h, TA_ERR_ARG, "ta_step: w, g and c must not be NULL");
+    if (!aligned16(w) || !aligned16(g) || !aligned16(c) || !aligned16(Hz))
+        return fail(h, TA_ERR_ALIGN, "ta_step: every device pointer must be 16-byte aligned");
+    if (step >= (1ull << 32)) return fail(h, TA_ERR_ARG, "ta_step: step must be below 2^32");
+    if (h->stepped && step <= h->last_step) return fail(h, TA_ERR_STATE, "ta_step: step must increase from call to call");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool bf16 = h->hp.grad_dtype == TA_GRAD_BF16;
+    const int P = Hz ? (int)h->hp.num_probes : 0;
+    const bool topk = h->topk && Hz;
+    DeviceBuffers &d = h->d;
+
+    const bool timed = h->timed_used < h->timed_cap;
+    cudaEvent_t *ev = timed ? &h->events[4 * (size_t)h->timed_used] : nullptr;
+    if (timed) cudaEventRecord(ev[0], s);
+
+    ta::SweepArgs sa{};
+    sa.items = d.items; sa.n_items = h->n_items; sa.n_batches = h->n_batches;
+    sa.g = g; sa.hz = Hz; sa.n_total = h->n_total; sa.seed = probe_seed; sa.step = (uint32_t)step;
+    sa.p_s1 = d.p_s1; sa.p_s2 = d.p_s2; sa.p_sa = d.p_sa;
+    sa.p_amax = d.p_amax; sa.p_amin = d.p_amin; sa.p_bad = d.p_bad;
+    sa.abs_s = d.abs_s; sa.hist = d.hist;
+    const bool ok = bf16 ? dispatch_sweep<true>(h, P, sa, s) : dispatch_sweep<false>(h, P, sa, s);
+    if (!ok) return fail(h, TA_ERR_ARG, "ta_step: unsupported probe count");
+    if (timed) cudaEventRecord(ev[1], s);
+
+    ta::DecideArgs da{};
+    da.item_lo = d.item_lo; da.seg_len = d.seg_len;
+    da.p_s1 = d.p_s1; da.p_s2 = d.p_s2; da.p_sa = d.p_sa;
+    da.p_amax = d.p_amax; da.p_amin = d.p_amin; da.p_bad = d.p_bad;
+    da.scratch = d.scratch; da.state = d.state; da.status = d.status;
+    da.hp = hyper_of(h->hp); da.eta0 = h->hp.eta0; da.L = h->L;
+    da.has_hz = Hz ? 1u : 0u; da.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; da.topk = topk ? 1u : 0u;
+    da.step = step;
+    ta::k_decide<<<h->L, ta::kThreads, 0, s>>>(da);
+    ++h->launches;
+
+    if (topk) {
+        const int grid = grid_for(h);
+        ta::SelectArgs se{d.hist, d.sel, d.state, d.seg_k, d.status};
+        ta::RefineArgs re{d.items, h->n_items, h->n_batches, d.abs_s, d.hist, d.sel, d.status};
+        ta::k_select<1><<<h->L, ta::kThreads, 0, s>>>(se);
+        ta::k_refine<2><<<grid, ta::kThreads, 0, s>>>(re);
+        ta::k_select<2><<<h->L, ta::kThreads, 0, s>>>(se);
+        ta::k_refine<3><<<grid, ta::kThreads, 0, s>>>(re);
+        ta::k_select<3><<<h->L, ta::kThreads, 0, s>>>(se);
+        const int zgrid = (int)std::min<uint64_t>((h->mask_words + ta::kThreads - 1) / ta::kThreads, (uint64_t)h->sm_count * 8);
+        ta::k_zero_mask<<<std::max(zgrid, 1), ta::kThreads, 0, s>>>(d.mask, h->mask_words, d.status);
+        ta::MaskArgs ma{d.items, h->n_items, h->n_batches, d.abs_s, d.mask, d.p_mass, d.sel, d.status};
+        ta::k_mask<<<grid, ta::kThreads, 0, s>>>(ma);
+        ta::FinishArgs fa{d.item_lo, d.items, d.seg_off, d.seg_len, d.abs_s, d.mask, d.p_mass, d.scratch, d.sel, d.state, d.status};
+        ta::k_finish<<<h->L, ta::kThreads, 0, s>>>(fa);
+        h->launches += 8;
+    }
+
+    if (timed) cudaEventRecord(ev[2], s);
+    ta::ApplyArgs aa{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status};
+    if (bf16) ta::k_apply<true><<<grid_for(h), ta::kThreads, 0, s>>>(aa);
+    else ta::k_apply<false><<<grid_for(h), ta::kThreads, 0, s>>>(aa);
+    ++h->launches;
+    if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
+
+    TA_CUDA(h, cudaGetLastError());
+    h->stepped = true;
+    h->last_step = step;
+    h->last_stream = s;
+    return TA_OK;
+}
+
+int ta_step_host(ta_handle *h, float *w_host, const void *g_host, const float *Hz_host, uint16_t *c_host,
+                 uint64_t probe_seed, uint64_t step, void *stream)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!w_host || !g_host || !c_host) return fail(h, TA_ERR_ARG, "ta_step_host: w, g and c must not be NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DeviceBuffers &d = h->d;
+    const size_t n = h->n_total;
+    const size_t g_bytes = n * (h->hp.grad_dtype == TA_GRAD_BF16 ? 2 : 4);
+    if (!d.st_w) {
+        TA_CUDA(h, dev_alloc(&d.st_w, n));
+        TA_CUDA(h, cudaMalloc(&d.st_g, std::max<size_t>(g_bytes, 16)));
+        TA_CUDA(h, dev_alloc(&d.st_c, n));
+        TA_CUDA(h, dev_alloc(&d.st_hz, n * h->hp.num_probes));
+    }
+    TA_CUDA(h, cudaMemcpyAsync(d.st_w, w_host, n * 4, cudaMemcpyHostToDevice, s));
+    TA_CUDA(h, cudaMemcpyAsync(d.st_g, g_host, g_bytes, cudaMemcpyHostToDevice, s));
+    if (Hz_host) TA_CUDA(h, cudaMemcpyAsync(d.st_hz, Hz_host, n * 4 * h->hp.num_probes, cudaMemcpyHostToDevice, s));
+    const int rc = ta_step(h, d.st_w, d.st_g, Hz_host ? d.st_hz : nullptr, d.st_c, probe_seed, step, stream);
+    if (rc != TA_OK) return rc;
+    // the new master weights of every layer, and the 16-bit copy of the layers that keep one
+    std::vector<ta::LayerState> st(h->L);
+    ta::Status status;
+    TA_CUDA(h, cudaMemcpyAsync(st.data(), d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost, s));
+    TA_CUDA(h, cudaMemcpyAsync(&status, d.status, sizeof(status), cudaMemcpyDeviceToHost, s));
+    TA_CUDA(h, cudaStreamSynchronize(s));
+    if (!status.skipped) {
+        const uint64_t first = h->table.front().offset, last = h->table.back().offset + h->table.back().length;
+        TA_CUDA(h, cudaMemcpyAsync(w_host + first, d.st_w + first, (last - first) * 4, cudaMemcpyDeviceToHost, s));
+        for (uint32_t l = 0; l < h->L;) {
+            if (st[l].code >= TA_CODE_FP32) { ++l; continue; }
+            uint32_t r = l;      // run of adjacent layers that keep a copy: one transfer (gaps hold stale staging data, so stop at gaps)
+            while (r + 1 < h->L && st[r + 1].code < TA_CODE_FP32 &&
+                   h->table[r + 1].offset == h->table[r].offset + h->table[r].length) ++r;
+            const uint64_t b = h->table[l].offset, e = h->table[r].offset + h->table[r].length;
+            TA_CUDA(h, cudaMemcpyAsync(c_host + b, d.st_c + b, (e - b) * 2, cudaMemcpyDeviceToHost, s));
+            l = r + 1;
+        }
+        TA_CUDA(h, cudaStreamSynchronize(s));
+    }
+    return TA_OK;
+}
+
+int ta_probe(ta_handle *h, uint64_t probe_seed, uint64_t step, uint32_t p, float *z_out, void *stream)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!z_out) return fail(h, TA_ERR_ARG, "ta_probe: z_out must not be NULL");
+    if (!aligned16(z_out)) return fail(h, TA_ERR_ALIGN, "ta_probe: z_out must be 16-byte aligned");
+    if (p >= h->hp.num_probes) return fail(h, TA_ERR_ARG, "ta_probe: p must be below num_probes");
+    if (step >= (1ull << 32)) return fail(h, TA_ERR_ARG, "ta_probe: step must be below 2^32");
+    const uint64_t n_vec = h->n_total / 4;
+    if (n_vec == 0) return TA_OK;
+    const int grid = (int)std::min<uint64_t>((n_vec + ta::kThreads - 1) / ta::kThreads, (uint64_t)h->sm_count * 16);
+    ta::k_probe<<<grid, ta::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(z_out, n_vec, probe_seed, (uint32_t)step, p);
+    ++h->launches;
+    TA_CUDA(h, cudaGetLastError());
+    return TA_OK;
+}
+
+int ta_stats(ta_handle *h, ta_layer_stats *out_host, ta_step_status *status)
+{
+    if (!h) return TA_ERR_ARG;
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    if (out_host) {
+        std::vector<ta::LayerState> st(h->L);
+        TA_CUDA(h, cudaMemcpy(st.data(), h->d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost));
+        for (uint32_t l = 0; l < h->L; ++l) {
+            ta_layer_stats &o = out_host[l];
+            o.grad_mean = (float)st[l].grad_mean;
+            o.grad_var = (float)st[l].grad_var;
+            o.ema_mean = st[l].ema_mean;
+            o.ema_var = st[l].ema_var;
+            o.lambda_max = st[l].lambda_max;
+            o.topk_threshold = st[l].thr;
+            o.topk_mass = (float)st[l].topk_mass;
+            o.eta_scale = st[l].eta_scale;
+            o.k = h->seg_k[l];
+            o.code = st[l].code;
+            o.near_threshold = st[l].near;
+        }
+    }
+    if (status) {
+        ta::Status s;
+        TA_CUDA(h, cudaMemcpy(&s, h->d.status, sizeof(s), cudaMemcpyDeviceToHost));
+        status->step = s.step;
+        status->nonfinite_count = s.nonfinite;
+        status->skipped = s.skipped;
+        status->near_threshold_count = s.near_count;
+    }
+    return TA_OK;
+}
+
+int ta_precision_codes(ta_handle *h, uint8_t *out_host)
+{
+    if (!h || !out_host) return TA_ERR_ARG;
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    std::vector<ta::LayerState> st(h->L);
+    TA_CUDA(h, cudaMemcpy(st.data(), h->d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost));
+    for (uint32_t l = 0; l < h->L; ++l) out_host[l] = (uint8_t)st[l].code;
+    return TA_OK;
+}
+
+int ta_masks(ta_handle *h, const uint32_t **dev_bits, uint64_t *num_words)
+{
+    if (!h || !dev_bits || !num_words) return TA_ERR_ARG;
+    *dev_bits = h->topk ? h->d.mask : nullptr;
+    *num_words = h->mask_words;
+    return TA_OK;
+}
+
+int ta_state_size(ta_handle *h, uint64_t *bytes)
+{
+    if (!h || !bytes) return TA_ERR_ARG;
+    *bytes = sizeof(StateHeader) + h->L * sizeof(ta::LayerState) + sizeof(ta::Status) + h->mask_words * sizeof(uint32_t);
+    return TA_OK;
+}
+
+int ta_state_save(ta_handle *h, void *buf_host, uint64_t bytes)
+{
+    uint64_t need = 0;
+    if (!h || !buf_host) return TA_ERR_ARG;
+    ta_state_size(h, &need);
+    if (bytes < need) return fail(h, TA_ERR_ARG, "ta_state_save: buffer too small");
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    char *p = static_cast<char *>(buf_host);
+    StateHeader hd{};
+    hd.magic = kStateMagic; hd.n_total = h->n_total; hd.last_step = h->last_step; hd.mask_words = h->mask_words;
+    hd.L = h->L; hd.stepped = h->stepped ? 1u : 0u; hd.hp = h->hp;
+    std::memcpy(p, &hd, sizeof(hd));
+    p += sizeof(hd);
+    TA_CUDA(h, cudaMemcpy(p, h->d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost));
+    p += h->L * sizeof(ta::LayerState);
+    TA_CUDA(h, cudaMemcpy(p, h->d.status, sizeof(ta::Status), cudaMemcpyDeviceToHost));
+    p += sizeof(ta::Status);
+    if (h->mask_words) TA_CUDA(h, cudaMemcpy(p, h->d.mask, h->mask_words * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    return TA_OK;
+}
+
+int ta_state_load(ta_handle *h, const void *buf_host, uint64_t bytes)
+{
+    uint64_t need = 0;
+    if (!h || !buf_host) return TA_ERR_ARG;
+    ta_state_size(h, &need);
+    if (bytes < need) return fail(h, TA_ERR_STATE, "ta_state_load: buffer smaller than this handle's state");
+    const char *p = static_cast<const char *>(buf_host);
+    StateHeader hd;
+    std::memcpy(&hd, p, sizeof(hd));
+    ta_hparams a = hd.hp, b = h->hp;
+    a.eta0 = b.eta0 = 0.f;     // the learning rate may differ: it is restored from the checkpoint
+    if (hd.magic != kStateMagic || hd.L != h->L || hd.n_total != h->n_total || hd.mask_words != h->mask_words ||
+        std::memcmp(&a, &b, sizeof(a)) != 0)
+        return fail(h, TA_ERR_STATE, "ta_state_load: checkpoint was written for another table or other hyper-parameters");
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    p += sizeof(hd);
+    TA_CUDA(h, cudaMemcpy(h->d.state, p, h->L * sizeof(ta::LayerState), cudaMemcpyHostToDevice));
+    p += h->L * sizeof(ta::LayerState);
+    TA_CUDA(h, cudaMemcpy(h->d.status, p, sizeof(ta::Status), cudaMemcpyHostToDevice));
+    p += sizeof(ta::Status);
+    if (h->mask_words) TA_CUDA(h, cudaMemcpy(h->d.mask, p, h->mask_words * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    h->hp.eta0 = hd.hp.eta0;
+    h->last_step = hd.last_step;
+    h->stepped = hd.stepped != 0;
+    return TA_OK;
+}
+
+int ta_batch_next(ta_batch_ctrl *bc, int64_t *B_next)
+{
+    if (!bc || !B_next) return TA_ERR_ARG;
+    if (!(bc->rho_low <= bc->rho_high) || bc->B_min > bc->B_max || bc->delta_up < 0 || bc->delta_down < 0) return TA_ERR_ARG;
+    uint64_t free_b = 0, total_b = 0;
+    ta_mem_reader rd = bc->mem_reader ? bc->mem_reader : default_mem_reader;
+    if (rd(bc->user, &free_b, &total_b) != 0 || free_b > total_b) return TA_ERR_CUDA;
+    const double usage = (double)(total_b - free_b);
+    const double mem_max = bc->mem_budget_bytes ? (double)bc->mem_budget_bytes : (double)total_b;
+    int64_t next = bc->B;
+    if (usage < bc->rho_low * mem_max) next = bc->B + bc->delta_up;          // Sec. 3.3, first case
+    else if (usage > bc->rho_high * mem_max) next = bc->B - bc->delta_down;  // second case
+    next = std::max(bc->B_min, std::min(bc->B_max, next));
+    bc->B = next;
+    *B_next = next;
+    return TA_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

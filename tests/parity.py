@@ -1,0 +1,157 @@
+"""Shared harness of the GPU parity tests: runs the CUDA library (through its C ABI binding) and the
+CPU oracle on the same seeded inputs and compares them element by element.
+
+Tolerances (the bar the method's specification sets):
+  codes, masks, k          bit-exact, except layers that either side flags as within 1e-5 relative
+                           of a decision threshold (those are returned as a list)
+  lambda_max, threshold,   bit-exact (the probe sums are exact sign flips added in one fixed order)
+  eta_scale
+  variance, EMA variance   1e-5 relative (+ 1e-12 * mean^2: float data cannot resolve less)
+  mean, EMA mean           1e-5 * max(|mean|, sqrt(var + mean^2))
+  master weights           <= 2 ulp (float);  16-bit copies <= 1 ulp of their format
+"""
+import numpy as np
+import torch
+
+import paper_2508_16905_b200 as ta
+from oracle import oracle as orc
+
+
+def ulp_f32(a, b):
+    ia = a.view(np.int32).astype(np.int64)
+    ib = b.view(np.int32).astype(np.int64)
+    ia = np.where(ia < 0, -(ia & 0x7FFFFFFF), ia)
+    ib = np.where(ib < 0, -(ib & 0x7FFFFFFF), ib)
+    return np.abs(ia - ib)
+
+
+def ulp_16(a, b):
+    ia = a.astype(np.int64)
+    ib = b.astype(np.int64)
+    ia = np.where(ia >= 0x8000, -(ia & 0x7FFF), ia)
+    ib = np.where(ib >= 0x8000, -(ib & 0x7FFF), ib)
+    return np.abs(ia - ib)
+
+
+def to_host_bits(t):
+    """torch tensor -> numpy; bfloat16 / float16 as uint16 bit patterns."""
+    if t.dtype in (torch.bfloat16, torch.float16):
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    if t.dtype == torch.int16:
+        return t.cpu().numpy().view(np.uint16)
+    return t.cpu().numpy()
+
+
+def segment_mask(table, n_total):
+    inside = np.zeros(n_total, dtype=bool)
+    for off, n in table:
+        inside[off:off + n] = True
+    return inside
+
+
+def oracle_hz(D_host, P, seed, t):
+    """Hz = D * z with the ORACLE's probes, [P * n_total] float32 on the host."""
+    n = D_host.size
+    return np.concatenate([D_host * orc.probe(seed, t, p, 0, n) for p in range(P)])
+
+
+def compare_stats(gl, ol, where=""):
+    """gl: ta_layer_stats, ol: oracle Layer.  Returns True when the layer is flagged near a threshold."""
+    mu, var = ol.grad_mean, ol.grad_var
+    scale = max(abs(mu), float(np.sqrt(var + mu * mu)))
+    assert abs(gl.grad_mean - mu) <= 1e-5 * scale + 1e-30, (where, "grad_mean", gl.grad_mean, mu)
+    assert abs(gl.grad_var - var) <= 1e-5 * var + 1e-12 * mu * mu + 1e-37, (where, "grad_var", gl.grad_var, var)
+    em, ev = ol.ema_mean, ol.ema_var
+    assert abs(gl.ema_var - ev) <= 1e-5 * abs(ev) + 1e-12 * em * em + 1e-37, (where, "ema_var", gl.ema_var, ev)
+    assert abs(gl.ema_mean - em) <= 1e-5 * max(abs(em), float(np.sqrt(abs(ev) + em * em))) + 1e-30, (where, "ema_mean")
+    assert np.float32(gl.lambda_max) == np.float32(ol.lambda_max), (where, "lambda_max", gl.lambda_max, ol.lambda_max)
+    assert np.float32(gl.topk_threshold) == np.float32(ol.topk_threshold), (where, "threshold", gl.topk_threshold, ol.topk_threshold)
+    assert gl.k == ol.k or ol.k == 0, (where, "k", gl.k, ol.k)
+    assert abs(gl.topk_mass - ol.topk_mass) <= 1e-5 * max(ol.topk_mass, 1e-30) or ol.k == 0, (where, "topk_mass", gl.topk_mass, ol.topk_mass)
+    near = bool(gl.near_threshold or ol.near_threshold)
+    if not near:
+        assert gl.code == ol.code, (where, "code", gl.code, ol.code)
+        assert np.float32(gl.eta_scale) == np.float32(ol.eta_scale), (where, "eta_scale", gl.eta_scale, ol.eta_scale)
+    return near
+
+
+class ParityRun:
+    """One workload on both sides.  `layers` restricts the oracle (and the comparison) to a subset of
+    the layers: layers are independent, so the oracle of a subset equals the full oracle on that subset."""
+
+    def __init__(self, table, n_total, hp, w0, layers=None):
+        self.table, self.n_total, self.hp = list(table), int(n_total), dict(hp)
+        self.layers = list(range(len(table))) if layers is None else list(layers)
+        self.sub_table = [self.table[l] for l in self.layers]
+        self.h = ta.ta_create(self.table, self.n_total, **self.hp)
+        self.o = orc.Oracle(self.sub_table, self.n_total, **self.hp)
+        self.w_dev = w0.to("cuda").clone()
+        self.c_dev = torch.full((self.n_total,), 0x5A5A, dtype=torch.int16, device="cuda")
+        self.w_host = to_host_bits(w0).copy()
+        self.c_host = np.full(self.n_total, 0x5A5A, dtype=np.uint16)
+        self.w_start = self.w_host.copy()
+        self.inside_all = segment_mask(self.table, self.n_total)
+        self.inside_sub = segment_mask(self.sub_table, self.n_total)
+        self.near_list = []
+        self.max_w_ulp = 0
+        self.max_c_ulp = 0
+
+    def step(self, t, g_dev, hz_host, seed, hz_dev=None, check=True):
+        """hz_host: oracle-side Hz (numpy [P*n_total]) or None; hz_dev defaults to a copy of hz_host."""
+        if hz_host is not None and hz_dev is None:
+            hz_dev = torch.from_numpy(hz_host).to("cuda")
+        ta.ta_step(self.h, self.w_dev, g_dev, hz_dev, self.c_dev, seed, t)
+        skipped = self.o.step(self.w_host, to_host_bits(g_dev), hz_host, self.c_host, seed, t)
+        if check:
+            self.check(t)
+        return skipped
+
+    def check(self, t):
+        stats, status = ta.ta_stats(self.h)
+        ost = self.o.status()
+        full = len(self.layers) == len(self.table)
+        if full:
+            assert (status.step, status.skipped, status.nonfinite_count) == (ost.step, ost.skipped, ost.nonfinite_count)
+        olayers = self.o.layers()
+        codes_gpu = ta.ta_precision_codes(self.h)
+        near_now = set()
+        for j, l in enumerate(self.layers):
+            if compare_stats(stats[l], olayers[j], where=f"step {t} layer {l}"):
+                near_now.add(l)
+                self.near_list.append((t, l, stats[l].code, olayers[j].code))
+            assert codes_gpu[l] == stats[l].code
+        w_gpu = self.w_dev.cpu().numpy()
+        c_gpu = to_host_bits(self.c_dev)
+        # gaps are never touched
+        assert np.array_equal(w_gpu[~self.inside_all].view(np.uint32), self.w_start[~self.inside_all].view(np.uint32))
+        assert np.all(c_gpu[~self.inside_all] == 0x5A5A)
+        for j, l in enumerate(self.layers):
+            off, n = self.table[l]
+            du = ulp_f32(w_gpu[off:off + n], self.w_host[off:off + n])
+            m = int(du.max())
+            self.max_w_ulp = max(self.max_w_ulp, m)
+            if stats[l].code != olayers[j].code or np.float32(stats[l].eta_scale) != np.float32(olayers[j].eta_scale):
+                assert l in near_now
+                # a listed near-threshold layer took another branch: resynchronise the oracle side to the GPU
+                self.w_host[off:off + n] = w_gpu[off:off + n]
+                self.c_host[off:off + n] = c_gpu[off:off + n]
+                continue
+            assert m <= 2, (t, l, "master weights differ by", m, "ulp")
+            dc = ulp_16(c_gpu[off:off + n], self.c_host[off:off + n])
+            mc = int(dc.max())
+            self.max_c_ulp = max(self.max_c_ulp, mc)
+            assert mc <= 1, (t, l, "16-bit copy differs by", mc, "ulp")
+        # masks
+        ppm = self.hp.get("topk_ppm", 1000000)
+        if ppm < 1000000:
+            mg = ta.ta_masks_to_host(self.h)
+            mo = self.o.mask()
+            if full:
+                assert np.array_equal(mg, mo), (t, "mask words differ", int((mg != mo).sum()))
+            else:
+                idx = np.flatnonzero(self.inside_sub)
+                bg = (mg[idx >> 5] >> (idx & 31).astype(np.uint32)) & 1
+                bo = (mo[idx >> 5] >> (idx & 31).astype(np.uint32)) & 1
+                assert np.array_equal(bg, bo)
+        else:
+            assert ta.ta_masks(self.h) == (None, 0)

@@ -1,0 +1,161 @@
+"""CPU-only checks of the boundary: the library loads, exports what the header declares, and the
+host-only parts (batch rule, argument validation that needs no device, replica bookkeeping) work."""
+import ctypes as C
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+import torch
+
+import paper_2508_16905_b200 as ta
+from paper_2508_16905_b200 import binding, workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "triaccel.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ta_[a-z_0-9]+)\s*\(", text)) - {"ta_mem_reader"})
+
+
+def test_library_exports_every_declared_symbol():
+    L = binding.lib()
+    names = declared_functions()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_struct_layouts_match_the_header():
+    assert C.sizeof(binding.ta_hparams) == 56
+    assert C.sizeof(binding.ta_layer_stats) == 48
+    assert C.sizeof(binding.ta_step_status) == 24
+    assert C.sizeof(binding.ta_segment) == 16
+
+
+def test_create_rejects_bad_arguments_before_touching_a_device():
+    bad = [
+        dict(table=[], n_total=8),
+        dict(table=[(0, 8), (4, 8)], n_total=16),                 # overlap
+        dict(table=[(8, 8), (0, 8)], n_total=16),                 # not ascending
+        dict(table=[(0, 0)], n_total=8),                          # empty layer
+        dict(table=[(0, 9)], n_total=8),                          # beyond n_total
+        dict(table=[(0, 6)], n_total=6),                          # n_total not a multiple of 4
+        dict(table=[(0, 8)], n_total=8, num_probes=3),
+        dict(table=[(0, 8)], n_total=8, topk_ppm=0),
+        dict(table=[(0, 8)], n_total=8, beta=1.0),
+        dict(table=[(0, 8)], n_total=8, t_ctrl=0),
+        dict(table=[(0, 8)], n_total=8, momentum=0.9),
+        dict(table=[(0, 8)], n_total=8, tau_low=2.0, tau_high=1.0),
+    ]
+    for kw in bad:
+        table, n_total = kw.pop("table"), kw.pop("n_total")
+        with pytest.raises(ta.TriAccelError) as e:
+            ta.ta_create(table, n_total, **kw)
+        assert e.value.code == ta.TA_ERR_ARG, kw
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")
+def test_no_device_means_a_loud_error_not_a_fallback():
+    with pytest.raises(ta.TriAccelError) as e:
+        ta.ta_create([(0, 8)], 8)
+    assert e.value.code == ta.TA_ERR_CUDA
+
+
+def _ctrl(B, free, total, budget=0, **kw):
+    state = {"calls": 0}
+
+    @binding.ta_mem_reader
+    def reader(user, free_p, total_p):
+        state["calls"] += 1
+        if free is None:
+            return 1
+        free_p[0], total_p[0] = free, total
+        return 0
+    args = dict(B=B, delta_up=8, delta_down=16, B_min=8, B_max=128, rho_low=0.7, rho_high=0.9)
+    args.update(kw)
+    bc = binding.ta_batch_ctrl(args["B"], args["delta_up"], args["delta_down"], args["B_min"], args["B_max"],
+                               args["rho_low"], args["rho_high"], budget, reader, None)
+    return bc, reader
+
+
+def test_batch_rule_truth_table_with_fake_reader():
+    # Sec. 3.3: usage = total - free
+    for B, used, want in [(96, 50, 104), (96, 95, 80), (96, 80, 96), (96, 70, 96), (96, 90, 96), (124, 10, 128), (16, 99, 8)]:
+        bc, keep = _ctrl(B, free=100 - used, total=100)
+        assert ta.ta_batch_next(bc) == want and bc.B == want
+    # a caller budget replaces the device total as MemMax
+    bc, keep = _ctrl(96, free=50, total=100, budget=50)       # usage 50 > 0.9 * 50
+    assert ta.ta_batch_next(bc) == 80
+    # the initial batch size of the paper's experiments grows while memory is free
+    bc, keep = _ctrl(96, free=90, total=100)
+    assert [ta.ta_batch_next(bc) for _ in range(5)] == [104, 112, 120, 128, 128]
+
+
+def test_batch_rule_errors():
+    bc, keep = _ctrl(96, free=None, total=0)
+    with pytest.raises(ta.TriAccelError) as e:
+        ta.ta_batch_next(bc)
+    assert e.value.code == ta.TA_ERR_CUDA and bc.B == 96
+    for kw in [dict(rho_low=0.95), dict(B_min=200), dict(delta_up=-1)]:
+        bc, keep = _ctrl(96, free=50, total=100, **kw)
+        with pytest.raises(ta.TriAccelError) as e:
+            ta.ta_batch_next(bc)
+        assert e.value.code == ta.TA_ERR_ARG
+
+
+def test_workload_tables_have_the_published_parameter_counts():
+    want = {"mlp_tiny": (4, 203530), "resnet18_cifar": (62, 11173962), "efficientnet_b0_cifar": (213, 4020358),
+            "resnet50_topk": (161, 25557032), "gpt_1p3b": (145, 1311080448)}
+    for name, (L, n) in want.items():
+        wl = W.get(name)
+        assert (len(wl.table), wl.num_params) == (L, n)
+        assert all(off % 8 == 0 for off, _ in wl.table) and wl.n_total % 8 == 0
+        ends = [o + n for o, n in wl.table]
+        assert all(wl.table[i + 1][0] >= ends[i] for i in range(L - 1)) and ends[-1] <= wl.n_total
+    small = [n for _, n in W.get("efficientnet_b0_cifar").table if n <= 1024]
+    assert (len(small), sum(small)) == (121, 33030)
+
+
+def test_generators_are_seeded_and_have_the_stated_distributions():
+    wl = W.get("mlp_tiny")
+    g1, g2 = W.make_grads(wl, 3), W.make_grads(wl, 3)
+    assert torch.equal(g1, g2) and not torch.equal(g1, W.make_grads(wl, 4))
+    for l, (off, n) in enumerate(wl.table[:3]):
+        assert float(g1[off:off + n].std()) == pytest.approx(1e-3 * 2 ** l, rel=0.2 if n < 1000 else 0.02)
+    D = W.make_curvature(wl)
+    assert float(D.min()) >= 1e-4 * 0.999 and float(D.max()) <= 1.0
+    assert float(torch.log(D).mean()) == pytest.approx(0.5 * torch.log(torch.tensor(1e-4)).item(), rel=0.02)
+    assert float(W.make_weights(wl).std()) == pytest.approx(0.05, rel=0.02)
+    heavy = W.get("resnet50_topk", shapes=W.resnet50_shapes(width=8))
+    g = W.make_grads(heavy, 1)
+    assert float((g.abs() > 8e-3).float().mean()) > 1e-4          # the Student-t(2) tail is present
+    assert W.make_grads(W.get("gpt_1p3b", shapes=W.gpt_shapes(layers=1, d=64, vocab=128)), 1).dtype == torch.bfloat16
+
+
+def test_replica_bookkeeping_world_size_2_gloo():
+    script = r"""
+import os, sys
+sys.path.insert(0, %r)
+from paper_2508_16905_b200 import dist as D
+rank, local_rank, world = D.init("gloo")
+assert world == 2
+D.barrier()
+ms, units = D.aggregate(10.0 + 5.0 * rank, 1000.0 * (rank + 1))
+assert (ms, units) == (15.0, 3000.0), (ms, units)
+D.barrier()
+D.shutdown()
+print("rank", rank, "ok")
+""" % ROOT
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
+    res = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                          "--master-addr", "127.0.0.1", "--master-port", "29571", "-c", script],
+                         capture_output=True, text=True, env=env, timeout=240)
+    if res.returncode != 0 and "-c" in res.stderr:
+        pytest.skip("torchrun cannot take -c here")
+    assert res.returncode == 0, res.stderr[-2000:]
+    assert res.stdout.count("ok") == 2
