@@ -146,6 +146,9 @@ def get(name, **overrides):
         w = dict(shapes=resnet50_shapes(), steps=50, num_probes=4, topk_ppm=100000, grad_recipe="heavy_tail")
     elif name == "gpt_1p3b":
         w = dict(shapes=gpt_shapes(), steps=20, grad_dtype="bf16", d_low=1e-6)
+    elif name == "gpt_1block":
+        # one decoder block plus the embedding: the 1.3B workload's tensor mix at a size a profiler can replay
+        w = dict(shapes=gpt_shapes(layers=1), steps=20, grad_dtype="bf16", d_low=1e-6)
     else:
         raise KeyError(name)
     w.update(overrides)
