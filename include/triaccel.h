@@ -239,6 +239,49 @@ typedef struct {
 
 int ta_batch_next(ta_batch_ctrl *bc, int64_t *B_next);
 
+/*
+ * ta_grad_moments_static -- per-layer gradient mean and population variance, computed without
+ * allocating anything.  (The paper has no counterpart: this entry point exists for the callers
+ * described next, not for a step of the method.)
+ *
+ * Who it is for: code that is not allowed to call cudaMalloc at the point where it needs the
+ * statistics -- a plug-in running inside a host application that owns all device memory and has
+ * handed out every byte of it, a callback that runs while an allocator lock is held, a process
+ * whose memory pool was sized up front and must not grow.  ta_create / ta_step allocate their
+ * workspace with cudaMalloc; this call never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * How: the scratch (one partial sum, sum of squares and non-finite count per tile of
+ * TA_STATIC_TILE_ELEMS gradient elements) lives in a fixed array inside the library's device
+ * image, about 640 KB, which every GPU that loads the library holds until the process exits.
+ * The layer table travels as a kernel argument.
+ *
+ *   table      host, L <= TA_STATIC_MAX_LAYERS segments, same rules as ta_create
+ *   g          device, float or bfloat16 per grad_dtype, 16-byte aligned, indexed by flat element
+ *   mean_var   device double[2 * L] (output): mean of layer l at [2l], variance at [2l + 1]
+ *   nonfinite  device uint32[L] (output) or NULL: non-finite gradient values per layer
+ *   stream     cudaStream_t as void*; the call is asynchronous
+ *
+ * Limits: the layers must fit in TA_STATIC_MAX_TILES tiles (tiles are cut on a global grid of
+ * TA_STATIC_TILE_ELEMS elements, so a layer of n elements needs about n / TA_STATIC_TILE_ELEMS + 1);
+ * that is roughly 536 million parameters.  A larger table is rejected with TA_ERR_ARG and a message
+ * (ta_static_last_error) and nothing is launched.
+ * The first call on each device looks up the device address of the array (cudaGetSymbolAddress, with
+ * that device current); make that first call outside any stream capture.
+ * All calls on one device share the one array and it keeps the previous call's contents.  Every
+ * slot a call reads is written earlier in the same call, so nothing needs clearing; but two calls
+ * whose kernels overlap on the GPU (different streams, no ordering between them) race on it and
+ * give wrong results.  Order them on one stream or with events.
+ * Results equal ta_stats().grad_mean / grad_var of a ta_step on the same gradient up to rounding
+ * (both accumulate in double).  Errors: TA_ERR_ARG, TA_ERR_ALIGN, TA_ERR_CUDA.
+ */
+#define TA_STATIC_TILE_ELEMS 16384u
+#define TA_STATIC_MAX_TILES  32768u
+#define TA_STATIC_MAX_LAYERS 128u
+int ta_grad_moments_static(const ta_segment *table, uint32_t L, const void *g, uint32_t grad_dtype,
+                           double *mean_var, uint32_t *nonfinite, void *stream);
+/* Message of the calling thread's last ta_grad_moments_static failure ("" if none). */
+const char *ta_static_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -19,7 +19,8 @@ TA_GRAD_F32, TA_GRAD_BF16 = 0, 1
 
 EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "ta_probe", "ta_stats",
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
-           "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end"]
+           "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
+           "ta_grad_moments_static", "ta_static_last_error"]
 
 
 class ta_segment(C.Structure):
@@ -90,8 +91,11 @@ def lib():
     L.ta_batch_next.argtypes = [C.POINTER(ta_batch_ctrl), C.POINTER(C.c_int64)]
     L.ta_timing_begin.argtypes = [vp, u32]
     L.ta_timing_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(u32)]
+    L.ta_grad_moments_static.argtypes = [C.POINTER(ta_segment), u32, vp, u32, vp, vp, vp]
+    L.ta_static_last_error.argtypes = []
+    L.ta_static_last_error.restype = C.c_char_p
     for name in EXPORTS:
-        if name != "ta_last_error":
+        if name not in ("ta_last_error", "ta_static_last_error"):
             getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -236,6 +240,18 @@ def ta_timing_end(h):
     a, b, c, n = C.c_double(), C.c_double(), C.c_double(), C.c_uint32()
     _check(lib().ta_timing_end(h.ptr, C.byref(a), C.byref(b), C.byref(c), C.byref(n)), h.ptr)
     return a.value, b.value, c.value, n.value
+
+
+def ta_grad_moments_static(table, g, grad_dtype, mean_var, nonfinite=None, stream=None):
+    """Per-layer gradient mean / variance through the entry point that allocates nothing.
+    table: sequence of (offset, length); g: CUDA tensor (float32 or bfloat16 per grad_dtype);
+    mean_var: CUDA float64 tensor [2 * L] (output); nonfinite: CUDA int32 tensor [L] or None."""
+    L = len(table)
+    segs = (ta_segment * max(L, 1))(*[ta_segment(int(o), int(n)) for o, n in table])
+    gd = {"f32": TA_GRAD_F32, "bf16": TA_GRAD_BF16}[grad_dtype] if isinstance(grad_dtype, str) else int(grad_dtype)
+    rc = lib().ta_grad_moments_static(segs, L, _dev_ptr(g), gd, _dev_ptr(mean_var), _dev_ptr(nonfinite), _stream(stream))
+    if rc != TA_OK:
+        raise TriAccelError(rc, (lib().ta_static_last_error() or b"").decode())
 
 
 def ta_state_save(h):
