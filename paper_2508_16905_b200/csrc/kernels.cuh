@@ -177,7 +177,10 @@ struct SweepArgs {
     // top-k only
     float *abs_s;             // [n_total] |S|
     uint32_t *hist;           // [L][kHistBins], level-1 histogram of |S| bit patterns
+    const uint32_t *batch_seg; // [n_batches] layer of a batch whose items all lie in one layer, else kMixedBatch
 };
+
+constexpr uint32_t kMixedBatch = 0xFFFFFFFFu;
 
 template <int P> struct RowData {
     float4 g;
@@ -240,14 +243,34 @@ __global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
     constexpr int PP = P > 0 ? P : 1;
     constexpr int U = (P <= 1) ? 8 : (P == 2 ? 4 : 2);     // rows in flight per lane
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
 
     for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
         const uint32_t it = batch * kWarps + warp;
-        if (it >= A.n_items) continue;
-        const Item item = A.items[it];
+        // a batch whose items share one layer counts its histogram in shared memory and flushes it once
+        bool uniform = false;
+        uint32_t batch_layer = 0;
+        if (TOPK) {
+            batch_layer = A.batch_seg[batch];
+            uniform = batch_layer != kMixedBatch;
+            if (uniform)
+                for (uint32_t b = threadIdx.x; b < (uint32_t)kHistBins; b += kThreads) sh_hist[b] = 0u;
+            __syncthreads();
+        }
+        const Item item = it < A.n_items ? A.items[it] : Item{0, 0, 0};
+        if (it < A.n_items && item.len == 0u && lane == 0) {   // padding item: neutral partials
+            A.p_s1[it] = 0.0; A.p_s2[it] = 0.0; A.p_bad[it] = 0u;
+            if (P > 0) { A.p_amax[it] = 0u; A.p_amin[it] = 0xFFFFFFFFu; }
+            if (TOPK) A.p_sa[it] = 0.0;
+        }
+        if (item.len != 0u) {
         const uint64_t begin = item.begin, end = begin + item.len;
         const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
         SweepAcc<P, TOPK> acc;
+        auto hist_add = [&](uint32_t ab) {
+            if (uniform) atomicAdd(&sh_hist[ab >> 20], 1u);
+            else atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
+        };
         uint32_t X[PP][4];
         uint64_t have_block = ~0ull;
 
@@ -280,7 +303,7 @@ __global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
                     const uint32_t ab = acc.element(GradVec<BF16>::load1(A.g, i), hv, sel, (k & 7u) * 4u + e);
                     if (TOPK) {
                         A.abs_s[i] = __uint_as_float(ab);
-                        atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
+                        hist_add(ab);
                     }
                 }
             }
@@ -306,7 +329,7 @@ __global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
                         }
                         const uint32_t ab = acc.element(gv[e], hv, sel, (k & 7u) * 4u + e);
                         av[e] = __uint_as_float(ab);
-                        if (TOPK) atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
+                        if (TOPK) hist_add(ab);
                     }
                     if (TOPK) {
                         const uint64_t i0 = (row + u) * 128ull + lane * 4u;
@@ -382,6 +405,16 @@ __global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
             A.p_bad[it] = bad;
             if (P > 0) { A.p_amax[it] = amax; A.p_amin[it] = amin; }
             if (TOPK) A.p_sa[it] = sa;
+        }
+        }   // item.len != 0
+        if (TOPK) {
+            __syncthreads();
+            if (uniform)
+                for (uint32_t b = threadIdx.x; b < (uint32_t)kHistBins; b += kThreads) {
+                    const uint32_t v = sh_hist[b];
+                    if (v) atomicAdd(A.hist + (uint64_t)batch_layer * kHistBins + b, v);
+                }
+            __syncthreads();
         }
     }
 }
@@ -539,6 +572,7 @@ __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
         const uint32_t it = batch * kWarps + warp;
         if (it >= A.n_items) continue;
         const Item item = A.items[it];
+        if (item.len == 0u) continue;
         const uint64_t begin = item.begin, end = begin + item.len;
         const float neg_eta = -A.state[item.seg].eta;
         const uint32_t code = A.state[item.seg].code;
@@ -625,127 +659,83 @@ __global__ void __launch_bounds__(kThreads) k_probe(float *z, uint64_t n_vec, ui
 }
 
 // ------------------------------------------------------------------ top-k: radix select on |S| bit patterns
+//
+// |S| >= 0, so the order of the values is the order of their 31-bit patterns.  Level 1 (bits 30..20)
+// is counted during the sweep.  k_select1 finds, per layer, the bin b1 that holds the k-th largest
+// value.  One more pass over |S| (k_mask_compact) sets the mask bits of every element in a bin above
+// b1 and appends the elements of bin b1 (value, index in layer) to the layer's candidate list.
+// k_resolve then finishes the selection on the candidates alone: two more value digits and, if more
+// candidates equal the threshold than are to be taken, three digits of the index (lower index first).
+// The result does not depend on the order in which candidates were appended.
+
+constexpr int kScanChunk = kHistBins / kThreads;
+
+// Whole block: the bin in which the `need`-th element falls when bins are walked from the top
+// (DESC) or from the bottom, and how many elements lie in the bins walked before it.
+template <bool DESC>
+__device__ __forceinline__ void block_find_bin(const uint32_t *h, int bins, uint32_t need, uint32_t *scan /*[kThreads]*/,
+                                               uint32_t *out /*[2]*/)
+{
+    const int tid = threadIdx.x, per = bins / kThreads;
+    uint32_t mine = 0;
+    for (int j = 0; j < per; ++j) {
+        const int pos = per * tid + j;
+        mine += h[DESC ? bins - 1 - pos : pos];
+    }
+    scan[tid] = mine;
+    __syncthreads();
+    for (int o = 1; o < kThreads; o <<= 1) {
+        const uint32_t add = tid >= o ? scan[tid - o] : 0u;
+        __syncthreads();
+        scan[tid] += add;
+        __syncthreads();
+    }
+    const uint32_t incl = scan[tid], before_me = incl - mine;
+    if (before_me < need && need <= incl) {
+        uint32_t cum = before_me;
+        for (int j = 0; j < per; ++j) {
+            const int pos = per * tid + j;
+            const int b = DESC ? bins - 1 - pos : pos;
+            const uint32_t cnt = h[b];
+            if (cum < need && need <= cum + cnt) { out[0] = (uint32_t)b; out[1] = cum; }
+            cum += cnt;
+        }
+    }
+    __syncthreads();
+}
 
 struct SelectArgs {
     uint32_t *hist;              // [L][kHistBins]
     SelectState *sel;            // [L]
-    LayerState *state;           // [L]
-    const uint64_t *seg_k;       // [L] mask population
+    uint32_t *cand_count;        // [L]
+    uint32_t *mask;
+    const uint64_t *seg_off, *seg_len, *seg_k;
     const Status *status;
 };
 
-// LEVEL 1: bits 30..20, LEVEL 2: bits 19..9, LEVEL 3: bits 8..0.  One block per layer: finds the
-// bin in which the k-th largest element falls and how many elements are still to be taken in it.
-template <int LEVEL>
-__global__ void __launch_bounds__(kThreads) k_select(const SelectArgs A)
+// One block per layer: level-1 bin of the k-th largest |S|; clears the histogram for the next step,
+// the candidate counter, and the (at most two) mask words the layer shares with a neighbour or a gap.
+__global__ void __launch_bounds__(kThreads) k_select1(const SelectArgs A)
 {
-    constexpr int BINS = LEVEL == 3 ? 512 : kHistBins;
-    constexpr int PER = BINS / kThreads;            // bins per thread, taken from the top down
-    __shared__ uint32_t h[BINS];
-    __shared__ uint32_t chunk[kThreads];
+    __shared__ uint32_t h[kHistBins];
+    __shared__ uint32_t scan[kThreads];
+    __shared__ uint32_t found[2];
     const uint32_t l = blockIdx.x, tid = threadIdx.x;
     uint32_t *gh = A.hist + (uint64_t)l * kHistBins;
-    for (int b = tid; b < BINS; b += kThreads) { h[b] = gh[b]; gh[b] = 0u; }
+    for (int b = tid; b < kHistBins; b += kThreads) { h[b] = gh[b]; gh[b] = 0u; }
     if (A.status->skipped) return;
     __syncthreads();
-    // thread t owns bins BINS-1-PER*t .. BINS-PER*(t+1), in descending order
-    uint32_t mine = 0;
-#pragma unroll
-    for (int j = 0; j < PER; ++j) mine += h[BINS - 1 - (PER * (int)tid + j)];
-    chunk[tid] = mine;
-    __syncthreads();
-    // inclusive scan over threads (Hillis-Steele)
-    for (int o = 1; o < kThreads; o <<= 1) {
-        const uint32_t add = tid >= (uint32_t)o ? chunk[tid - o] : 0u;
-        __syncthreads();
-        chunk[tid] += add;
-        __syncthreads();
-    }
-    const uint32_t need = LEVEL == 1 ? (uint32_t)A.seg_k[l] : A.sel[l].remaining;
-    const uint32_t above = chunk[tid] - mine;       // elements in bins above this thread's bins
-    if (above < need && need <= chunk[tid]) {
-        uint32_t cum = above;
-#pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            const int b = BINS - 1 - (PER * (int)tid + j);
-            const uint32_t cnt = h[b];
-            if (cum < need && need <= cum + cnt) {
-                SelectState s = A.sel[l];
-                s.prefix = LEVEL == 1 ? (uint32_t)b : ((s.prefix << (LEVEL == 3 ? 9 : 11)) | (uint32_t)b);
-                s.remaining = need - cum;
-                if (LEVEL == 3) {
-                    s.thr_bits = s.prefix;
-                    s.take_equal = s.remaining;
-                    s.surplus = cnt > s.remaining ? 1u : 0u;
-                    A.state[l].thr = __uint_as_float(s.thr_bits);
-                }
-                A.sel[l] = s;
-            }
-            cum += cnt;
-        }
-    }
-}
-
-struct RefineArgs {
-    const Item *items;
-    uint32_t n_items, n_batches;
-    const float *abs_s;
-    uint32_t *hist;
-    const SelectState *sel;
-    const Status *status;
-};
-
-// Histogram of the next digit over the elements whose higher bits equal the layer's prefix.
-template <int LEVEL>
-__global__ void __launch_bounds__(kThreads) k_refine(const RefineArgs A)
-{
-    if (A.status->skipped) return;
-    constexpr int SHIFT_PREFIX = LEVEL == 2 ? 20 : 9;
-    constexpr int SHIFT_DIGIT = LEVEL == 2 ? 9 : 0;
-    constexpr uint32_t DIGIT_MASK = LEVEL == 2 ? 2047u : 511u;
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
-        const uint32_t it = batch * kWarps + warp;
-        if (it >= A.n_items) continue;
-        const Item item = A.items[it];
-        const uint64_t begin = item.begin, end = begin + item.len;
-        const uint32_t prefix = A.sel[item.seg].prefix;
-        uint32_t *hist = A.hist + (uint64_t)item.seg * kHistBins;
-        const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
-        for (uint64_t row = row_first; row <= row_last; ++row) {
-            const uint64_t i0 = row * 128ull + lane * 4u;
-            const bool full = row * 128ull >= begin && row * 128ull + 128u <= end;
-            uint32_t ab[4];
-            bool ok[4];
-            if (full) {
-                const float4 v = __ldg(reinterpret_cast<const float4 *>(A.abs_s + i0));
-                ab[0] = __float_as_uint(v.x); ab[1] = __float_as_uint(v.y);
-                ab[2] = __float_as_uint(v.z); ab[3] = __float_as_uint(v.w);
-                ok[0] = ok[1] = ok[2] = ok[3] = true;
-            } else {
-                for (uint32_t e = 0; e < 4; ++e) {
-                    ok[e] = i0 + e >= begin && i0 + e < end;
-                    ab[e] = ok[e] ? __float_as_uint(A.abs_s[i0 + e]) : 0u;
-                }
-            }
-#pragma unroll
-            for (uint32_t e = 0; e < 4; ++e) {
-                const bool hit = ok[e] && (ab[e] >> SHIFT_PREFIX) == prefix;
-                const uint32_t digit = (ab[e] >> SHIFT_DIGIT) & DIGIT_MASK;
-                // the whole warp is converged here: aggregate the common case of one shared digit
-                const uint32_t m = __ballot_sync(0xFFFFFFFFu, hit);
-                if (m) {
-                    const int leader = __ffs(m) - 1;
-                    const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, leader);
-                    const uint32_t same = __ballot_sync(0xFFFFFFFFu, hit && digit == d0);
-                    if (same == m) {
-                        if ((int)lane == leader) atomicAdd(hist + d0, (uint32_t)__popc(m));
-                    } else if (hit) {
-                        atomicAdd(hist + digit, 1u);
-                    }
-                }
-            }
-        }
+    block_find_bin<true>(h, kHistBins, (uint32_t)A.seg_k[l], scan, found);
+    if (tid == 0) {
+        SelectState s;
+        s.prefix = found[0];
+        s.remaining = (uint32_t)A.seg_k[l] - found[1];
+        s.thr_bits = 0u; s.take_equal = 0u; s.surplus = 0u; s.pad = 0u;
+        A.sel[l] = s;
+        A.cand_count[l] = 0u;
+        const uint64_t b = A.seg_off[l], e = b + A.seg_len[l];
+        if (b & 31u) A.mask[b >> 5] = 0u;
+        if (e & 31u) A.mask[e >> 5] = 0u;
     }
 }
 
@@ -754,21 +744,16 @@ struct MaskArgs {
     uint32_t n_items, n_batches;
     const float *abs_s;
     uint32_t *mask;
-    double *p_mass;              // per item: sum of |S| strictly above the threshold
+    double *p_mass;              // per item: sum of |S| in bins above the layer's level-1 bin
     const SelectState *sel;
+    const uint64_t *seg_off, *seg_len;
+    uint32_t *cand_count;        // [L]
+    uint32_t *cand_val;          // [n_total], candidates of layer l at seg_off[l] ...
+    uint32_t *cand_idx;          // [n_total]
     const Status *status;
 };
 
-__global__ void __launch_bounds__(kThreads) k_zero_mask(uint32_t *mask, uint64_t words, const Status *status)
-{
-    if (status->skipped) return;
-    for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < words; i += (uint64_t)gridDim.x * blockDim.x)
-        mask[i] = 0u;
-}
-
-// Sets the bit of every element above the threshold, and of those equal to it when all of them
-// belong to the mask; a layer with surplus ties gets its equal elements from k_finish.
-__global__ void __launch_bounds__(kThreads) k_mask(const MaskArgs A)
+__global__ void __launch_bounds__(kThreads) k_mask_compact(const MaskArgs A)
 {
     if (A.status->skipped) return;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -776,101 +761,192 @@ __global__ void __launch_bounds__(kThreads) k_mask(const MaskArgs A)
         const uint32_t it = batch * kWarps + warp;
         if (it >= A.n_items) continue;
         const Item item = A.items[it];
+        if (item.len == 0u) { if (lane == 0) A.p_mass[it] = 0.0; continue; }
         const uint64_t begin = item.begin, end = begin + item.len;
-        const SelectState s = A.sel[item.seg];
-        const uint32_t ge = s.surplus ? s.thr_bits + 1u : s.thr_bits;   // take bit patterns >= ge
+        const uint64_t seg_b = A.seg_off[item.seg], seg_e = seg_b + A.seg_len[item.seg];
+        const uint32_t b1 = A.sel[item.seg].prefix;
+        uint32_t *cval = A.cand_val + seg_b, *cidx = A.cand_idx + seg_b;
         double mass = 0.0;
         const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
-        for (uint64_t row = row_first; row <= row_last; ++row) {
-            const uint64_t i0 = row * 128ull + lane * 4u;
-            const bool full = row * 128ull >= begin && row * 128ull + 128u <= end;
-            uint32_t nib = 0u;
-            if (full) {
-                const float4 v = __ldcs(reinterpret_cast<const float4 *>(A.abs_s + i0));
-                const float av[4] = {v.x, v.y, v.z, v.w};
+        constexpr int U = 4;
+        uint64_t row = row_first;
+        while (row <= row_last) {
+            const bool group_full = row * 128ull >= begin && (row + U) * 128ull <= end;
+            const int rows = group_full ? U : 1;
+            float4 v[U];
+            bool full = group_full;
+            if (group_full) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) v[u] = __ldcs(reinterpret_cast<const float4 *>(A.abs_s + (row + u) * 128ull + lane * 4u));
+            } else {
+                full = row * 128ull >= begin && row * 128ull + 128u <= end;
+                if (full) v[0] = __ldcs(reinterpret_cast<const float4 *>(A.abs_s + row * 128ull + lane * 4u));
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (u >= rows) break;
+                const uint64_t i0 = (row + u) * 128ull + lane * 4u;
+                uint32_t ab[4];
+                bool ok[4];
+                if (full) {
+                    ab[0] = __float_as_uint(v[u].x); ab[1] = __float_as_uint(v[u].y);
+                    ab[2] = __float_as_uint(v[u].z); ab[3] = __float_as_uint(v[u].w);
+                    ok[0] = ok[1] = ok[2] = ok[3] = true;
+                } else {
+#pragma unroll
+                    for (uint32_t e = 0; e < 4; ++e) {
+                        ok[e] = i0 + e >= begin && i0 + e < end;
+                        ab[e] = ok[e] ? __float_as_uint(A.abs_s[i0 + e]) : 0u;
+                    }
+                }
+                uint32_t nib = 0u, cand = 0u;
 #pragma unroll
                 for (uint32_t e = 0; e < 4; ++e) {
-                    const uint32_t ab = __float_as_uint(av[e]);
-                    if (ab >= ge) nib |= 1u << e;
-                    if (ab > s.thr_bits) mass += (double)av[e];
+                    const uint32_t bin = ab[e] >> 20;
+                    if (ok[e] && bin > b1) { nib |= 1u << e; mass += (double)__uint_as_float(ab[e]); }
+                    if (ok[e] && bin == b1) cand |= 1u << e;
                 }
-            } else {
-                for (uint32_t e = 0; e < 4; ++e) {
-                    if (i0 + e >= begin && i0 + e < end) {
-                        const float a = A.abs_s[i0 + e];
-                        const uint32_t ab = __float_as_uint(a);
-                        if (ab >= ge) nib |= 1u << e;
-                        if (ab > s.thr_bits) mass += (double)a;
+                // candidates: one slot reservation per warp and row
+                const uint32_t n_mine = (uint32_t)__popc(cand);
+                uint32_t incl = n_mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if ((int)lane >= o) incl += t;
+                }
+                const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (total) {
+                    uint32_t base = 0;
+                    if (lane == 31) base = atomicAdd(A.cand_count + item.seg, total);
+                    base = __shfl_sync(0xFFFFFFFFu, base, 31) + incl - n_mine;
+#pragma unroll
+                    for (uint32_t e = 0; e < 4; ++e)
+                        if (cand & (1u << e)) { cval[base] = ab[e]; cidx[base] = (uint32_t)(i0 + e - seg_b); ++base; }
+                }
+                // mask words: 8 lanes make one 32-bit word
+                uint32_t word = nib << ((lane & 7u) * 4u);
+                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+                if ((lane & 7u) == 0u) {
+                    const uint64_t w0 = (row + u) * 128ull + (lane >> 3) * 32ull;     // first element of this word
+                    uint32_t *dst = A.mask + (w0 >> 5);
+                    if (w0 >= begin && w0 + 32u <= end) {
+                        *dst = word;                          // the word lies entirely inside this item
+                    } else if (w0 + 32u > begin && w0 < end) {
+                        // cut by the layer's first or last element (items are cut on multiples of 128 inside a
+                        // layer): the word is shared with a neighbour or a gap and was cleared by k_select1
+                        if (word) atomicOr(dst, word);
                     }
                 }
             }
-            uint32_t word = nib << ((lane & 7u) * 4u);
-            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
-            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
-            if ((lane & 7u) == 0u) {
-                uint32_t *dst = A.mask + (row * 4ull + (lane >> 3));
-                if (full) *dst = word;
-                else if (word) atomicOr(dst, word);
-            }
+            row += rows;
         }
         mass = warp_sum(mass);
         if (lane == 0) A.p_mass[it] = mass;
     }
 }
 
-struct FinishArgs {
+struct ResolveArgs {
     const uint32_t *item_lo;
-    const ta::Item *items;
     const uint64_t *seg_off, *seg_len;
-    const float *abs_s;
+    const uint32_t *cand_count, *cand_val, *cand_idx;
     uint32_t *mask;
     const double *p_mass;
     const LayerScratch *scratch;
-    const SelectState *sel;
+    SelectState *sel;
     LayerState *state;
     const Status *status;
 };
 
-// One block per layer: the masked share of |S|, and, for a layer with surplus ties at the
-// threshold, the bits of the first take_equal elements equal to it, in index order.
-__global__ void __launch_bounds__(kThreads) k_finish(const FinishArgs A)
+// One block per layer: finishes the selection among the layer's candidates.
+__global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
 {
     if (A.status->skipped) return;
+    __shared__ uint32_t h[kHistBins];
+    __shared__ uint32_t scan[kThreads];
+    __shared__ uint32_t found[2];
     __shared__ double red[kWarps];
-    __shared__ uint32_t wsum[kWarps];
-    const uint32_t l = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    const SelectState s = A.sel[l];
+    __shared__ unsigned long long acc_u64[2];
+    const uint32_t l = blockIdx.x, tid = threadIdx.x;
+    const uint64_t off = A.seg_off[l];
+    const uint32_t m = A.cand_count[l];
+    const uint32_t *cv = A.cand_val + off, *ci = A.cand_idx + off;
+    SelectState s = A.sel[l];
+    const uint32_t b1 = s.prefix;
+
+    auto clear = [&](int bins) { for (int b = tid; b < bins; b += kThreads) h[b] = 0u; __syncthreads(); };
+
+    // value digits: bits 19..9, then bits 8..0
+    clear(kHistBins);
+    for (uint32_t j = tid; j < m; j += kThreads) atomicAdd(&h[(cv[j] >> 9) & 2047u], 1u);
+    __syncthreads();
+    block_find_bin<true>(h, kHistBins, s.remaining, scan, found);
+    const uint32_t b2 = found[0], r2 = s.remaining - found[1];
+    const uint32_t pre22 = (b1 << 11) | b2;
+    __syncthreads();
+    clear(512);
+    for (uint32_t j = tid; j < m; j += kThreads) { const uint32_t v = cv[j]; if ((v >> 9) == pre22) atomicAdd(&h[v & 511u], 1u); }
+    __syncthreads();
+    block_find_bin<true>(h, 512, r2, scan, found);
+    const uint32_t thr = (pre22 << 9) | found[0];
+    const uint32_t take_equal = r2 - found[1];
+    const uint32_t n_equal = h[found[0]];
+    __syncthreads();
+
+    // index digits (only when ties at the threshold exceed what is taken): bits 31..21, 20..10, 9..0
+    uint32_t idx_limit = 0xFFFFFFFFu;           // equal-valued candidates with index <= idx_limit are taken
+    if (n_equal > take_equal) {
+        uint32_t need = take_equal, prefix = 0u;
+        const int shifts[3] = {21, 10, 0};
+        const int widths[3] = {11, 11, 10};
+        for (int lev = 0; lev < 3; ++lev) {
+            const int bins = 1 << widths[lev];
+            clear(kHistBins);
+            for (uint32_t j = tid; j < m; j += kThreads) {
+                if (cv[j] != thr) continue;
+                const uint32_t ix = ci[j];
+                const bool match = lev == 0 ? true : (ix >> (shifts[lev] + widths[lev])) == prefix;
+                if (match) atomicAdd(&h[(ix >> shifts[lev]) & (uint32_t)(bins - 1)], 1u);
+            }
+            __syncthreads();
+            block_find_bin<false>(h, lev == 2 ? 1024 : kHistBins, need, scan, found);
+            prefix = (prefix << widths[lev]) | found[0];
+            need -= found[1];
+            __syncthreads();
+        }
+        idx_limit = prefix;
+    }
+
+    // set the bits of the taken candidates; their sum is exact: all share sign and exponent
+    // (the exponent is part of the level-1 digit), so it is count * 2^e + (sum of mantissas) * 2^(e-23)
+    unsigned long long cnt = 0ull, mant = 0ull;
+    for (uint32_t j = tid; j < m; j += kThreads) {
+        const uint32_t v = cv[j], ix = ci[j];
+        if (v > thr || (v == thr && ix <= idx_limit)) {
+            const uint64_t i = off + ix;
+            atomicOr(A.mask + (i >> 5), 1u << (i & 31u));
+            ++cnt;
+            mant += v & 0x007FFFFFu;
+        }
+    }
+    if (tid < 2) acc_u64[tid] = 0ull;
+    __syncthreads();
+    atomicAdd(&acc_u64[0], cnt);
+    atomicAdd(&acc_u64[1], mant);
     double mass = 0.0;
     for (uint32_t i = A.item_lo[l] + tid; i < A.item_lo[l + 1]; i += kThreads) mass += A.p_mass[i];
     mass = block_sum(mass, red);
     if (tid == 0) {
+        const uint32_t expo = (b1 >> 3) & 0xFFu;                      // level-1 digit = 8 exponent bits + 3 mantissa bits
+        const double unit = expo ? ldexp(1.0, (int)expo - 127 - 23) : ldexp(1.0, -126 - 23);
+        const double cand_sum = expo ? ((double)acc_u64[0] * 8388608.0 + (double)acc_u64[1]) * unit
+                                     : (double)acc_u64[1] * unit;
         const double all = A.scratch[l].sum_abs;
-        const double masked = mass + (double)s.take_equal * (double)__uint_as_float(s.thr_bits);
-        A.state[l].topk_mass = all > 0.0 ? masked / all : 1.0;
-    }
-    if (!s.surplus) return;
-    const uint64_t off = A.seg_off[l], n = A.seg_len[l];
-    uint32_t taken = 0;
-    for (uint64_t base = 0; base < n && taken < s.take_equal; base += kThreads) {
-        const uint64_t j = base + tid;
-        const bool eq = j < n && __float_as_uint(A.abs_s[off + j]) == s.thr_bits;
-        const uint32_t m = __ballot_sync(0xFFFFFFFFu, eq);
-        __syncthreads();
-        if (lane == 0) wsum[warp] = (uint32_t)__popc(m);
-        __syncthreads();
-        uint32_t before = 0, total = 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            if (w < (int)warp) before += wsum[w];
-            total += wsum[w];
-        }
-        const uint32_t rank = taken + before + (uint32_t)__popc(m & ((1u << lane) - 1u));
-        if (eq && rank < s.take_equal) {
-            const uint64_t i = off + j;
-            atomicOr(A.mask + (i >> 5), 1u << (i & 31u));
-        }
-        taken += total;
+        s.thr_bits = thr; s.take_equal = take_equal; s.surplus = n_equal > take_equal ? 1u : 0u;
+        A.sel[l] = s;
+        A.state[l].thr = __uint_as_float(thr);
+        A.state[l].topk_mass = all > 0.0 ? (mass + cand_sum) / all : 1.0;
     }
 }
 

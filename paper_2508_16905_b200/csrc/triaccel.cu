@@ -28,6 +28,7 @@ struct DeviceBuffers {
     uint32_t *hist = nullptr;
     ta::SelectState *sel = nullptr;
     uint32_t *mask = nullptr;
+    uint32_t *cand_count = nullptr, *cand_val = nullptr, *cand_idx = nullptr, *batch_seg = nullptr;
     // host-tensor staging (ta_step_host)
     float *st_w = nullptr, *st_hz = nullptr;
     void *st_g = nullptr;
@@ -84,7 +85,7 @@ template <typename T> cudaError_t dev_alloc(T **p, size_t count)
 void free_all(DeviceBuffers &d)
 {
     void *ptrs[] = {d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
-                    d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.st_w, d.st_hz,
+                    d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
     for (void *p : ptrs)
         if (p) cudaFree(p);
@@ -241,6 +242,12 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         seg_len[l] = table[l].length;
         uint64_t k = (table[l].length * (uint64_t)hp->topk_ppm + 999999ull) / 1000000ull;
         h->seg_k[l] = k < 1 ? 1 : k;
+        // top-k: a layer of at least one full batch starts on a batch boundary, so that its batches hold one
+        // layer only and can count their histogram in shared memory (padding items are empty)
+        const uint64_t layer_items = (e - 1) / h->item_elems - b / h->item_elems + 1;
+        if (h->topk && layer_items >= (uint64_t)ta::kWarps && l > 0)
+            while (items.size() % ta::kWarps) items.push_back(ta::Item{b, 0u, l - 1});
+        item_lo[l] = (uint32_t)items.size();
         for (uint64_t p = b; p < e;) {
             const uint64_t next = std::min(e, (p / h->item_elems + 1) * (uint64_t)h->item_elems);
             items.push_back(ta::Item{p, (uint32_t)(next - p), l});
@@ -251,6 +258,17 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     item_lo[L] = (uint32_t)items.size();
     h->n_items = (uint32_t)items.size();
     h->n_batches = (h->n_items + ta::kWarps - 1) / ta::kWarps;
+    std::vector<uint32_t> batch_seg(h->n_batches, ta::kMixedBatch);
+    for (uint32_t bt = 0; bt < h->n_batches; ++bt) {
+        uint32_t seg = ta::kMixedBatch;
+        bool uniform = true;
+        for (uint32_t i = bt * ta::kWarps; i < std::min(h->n_items, (bt + 1) * ta::kWarps); ++i) {
+            if (items[i].len == 0) continue;
+            if (seg == ta::kMixedBatch) seg = items[i].seg;
+            else if (seg != items[i].seg) uniform = false;
+        }
+        batch_seg[bt] = uniform ? seg : ta::kMixedBatch;
+    }
 
     DeviceBuffers &d = h->d;
     TA_TRY(dev_alloc(&d.items, items.size()));
@@ -273,6 +291,12 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         TA_TRY(dev_alloc(&d.hist, (size_t)L * ta::kHistBins));
         TA_TRY(dev_alloc(&d.sel, L));
         TA_TRY(dev_alloc(&d.mask, h->mask_words));
+        TA_TRY(dev_alloc(&d.cand_count, L));
+        TA_TRY(dev_alloc(&d.cand_val, n_total));
+        TA_TRY(dev_alloc(&d.cand_idx, n_total));
+        TA_TRY(dev_alloc(&d.batch_seg, h->n_batches));
+        TA_TRY(cudaMemset(d.cand_count, 0, (size_t)L * sizeof(uint32_t)));
+        TA_TRY(cudaMemcpy(d.batch_seg, batch_seg.data(), batch_seg.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
         TA_TRY(cudaMemset(d.hist, 0, (size_t)L * ta::kHistBins * sizeof(uint32_t)));
         TA_TRY(cudaMemset(d.sel, 0, (size_t)L * sizeof(ta::SelectState)));
         TA_TRY(cudaMemset(d.mask, 0, h->mask_words * sizeof(uint32_t)));
@@ -384,7 +408,7 @@ int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
     sa.g = g; sa.hz = Hz; sa.n_total = h->n_total; sa.seed = probe_seed; sa.step = (uint32_t)step;
     sa.p_s1 = d.p_s1; sa.p_s2 = d.p_s2; sa.p_sa = d.p_sa;
     sa.p_amax = d.p_amax; sa.p_amin = d.p_amin; sa.p_bad = d.p_bad;
-    sa.abs_s = d.abs_s; sa.hist = d.hist;
+    sa.abs_s = d.abs_s; sa.hist = d.hist; sa.batch_seg = d.batch_seg;
     const bool ok = bf16 ? dispatch_sweep<true>(h, P, sa, s) : dispatch_sweep<false>(h, P, sa, s);
     if (!ok) return fail(h, TA_ERR_ARG, "ta_step: unsupported probe count");
     if (timed) cudaEventRecord(ev[1], s);
@@ -402,20 +426,15 @@ int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
 
     if (topk) {
         const int grid = grid_for(h);
-        ta::SelectArgs se{d.hist, d.sel, d.state, d.seg_k, d.status};
-        ta::RefineArgs re{d.items, h->n_items, h->n_batches, d.abs_s, d.hist, d.sel, d.status};
-        ta::k_select<1><<<h->L, ta::kThreads, 0, s>>>(se);
-        ta::k_refine<2><<<grid, ta::kThreads, 0, s>>>(re);
-        ta::k_select<2><<<h->L, ta::kThreads, 0, s>>>(se);
-        ta::k_refine<3><<<grid, ta::kThreads, 0, s>>>(re);
-        ta::k_select<3><<<h->L, ta::kThreads, 0, s>>>(se);
-        const int zgrid = (int)std::min<uint64_t>((h->mask_words + ta::kThreads - 1) / ta::kThreads, (uint64_t)h->sm_count * 8);
-        ta::k_zero_mask<<<std::max(zgrid, 1), ta::kThreads, 0, s>>>(d.mask, h->mask_words, d.status);
-        ta::MaskArgs ma{d.items, h->n_items, h->n_batches, d.abs_s, d.mask, d.p_mass, d.sel, d.status};
-        ta::k_mask<<<grid, ta::kThreads, 0, s>>>(ma);
-        ta::FinishArgs fa{d.item_lo, d.items, d.seg_off, d.seg_len, d.abs_s, d.mask, d.p_mass, d.scratch, d.sel, d.state, d.status};
-        ta::k_finish<<<h->L, ta::kThreads, 0, s>>>(fa);
-        h->launches += 8;
+        ta::SelectArgs se{d.hist, d.sel, d.cand_count, d.mask, d.seg_off, d.seg_len, d.seg_k, d.status};
+        ta::k_select1<<<h->L, ta::kThreads, 0, s>>>(se);
+        ta::MaskArgs ma{d.items, h->n_items, h->n_batches, d.abs_s, d.mask, d.p_mass, d.sel, d.seg_off, d.seg_len,
+                        d.cand_count, d.cand_val, d.cand_idx, d.status};
+        ta::k_mask_compact<<<grid, ta::kThreads, 0, s>>>(ma);
+        ta::ResolveArgs ra{d.item_lo, d.seg_off, d.seg_len, d.cand_count, d.cand_val, d.cand_idx, d.mask, d.p_mass,
+                           d.scratch, d.sel, d.state, d.status};
+        ta::k_resolve<<<h->L, ta::kThreads, 0, s>>>(ra);
+        h->launches += 3;
     }
 
     if (timed) cudaEventRecord(ev[2], s);
