@@ -421,6 +421,41 @@ __global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
 
 // ------------------------------------------------------------------ decisions
 
+// Whole block: the bin in which the `need`-th element falls when bins are walked from the top
+// (DESC) or from the bottom, and how many elements lie in the bins walked before it.
+template <bool DESC>
+__device__ __forceinline__ void block_find_bin(const uint32_t *h, int bins, uint32_t need, uint32_t *scan /*[kThreads]*/,
+                                               uint32_t *out /*[2]*/)
+{
+    const int tid = threadIdx.x, per = bins / kThreads;
+    uint32_t mine = 0;
+    for (int j = 0; j < per; ++j) {
+        const int pos = per * tid + j;
+        mine += h[DESC ? bins - 1 - pos : pos];
+    }
+    scan[tid] = mine;
+    __syncthreads();
+    for (int o = 1; o < kThreads; o <<= 1) {
+        const uint32_t add = tid >= o ? scan[tid - o] : 0u;
+        __syncthreads();
+        scan[tid] += add;
+        __syncthreads();
+    }
+    const uint32_t incl = scan[tid], before_me = incl - mine;
+    if (before_me < need && need <= incl) {
+        uint32_t cum = before_me;
+        for (int j = 0; j < per; ++j) {
+            const int pos = per * tid + j;
+            const int b = DESC ? bins - 1 - pos : pos;
+            const uint32_t cnt = h[b];
+            if (cum < need && need <= cum + cnt) { out[0] = (uint32_t)b; out[1] = cum; }
+            cum += cnt;
+        }
+    }
+    __syncthreads();
+}
+
+
 struct DecideArgs {
     const uint32_t *item_lo;        // [L + 1] first item of each layer
     const uint64_t *seg_len;        // [L]
@@ -434,6 +469,11 @@ struct DecideArgs {
     uint32_t L;
     uint32_t has_hz, control, topk;
     unsigned long long step;
+    // top-k only: level-1 histogram [L][kHistBins], selection bookkeeping, candidate counters, mask population
+    uint32_t *hist;
+    SelectState *sel;
+    uint32_t *cand_count;
+    const uint64_t *seg_k;
 };
 
 // Reads another block's results past the L1 cache (they were published with a fence).
@@ -487,8 +527,28 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     __shared__ double red[kWarps];
     __shared__ uint32_t red_u[2][kWarps];
     __shared__ uint32_t is_last;
+    __shared__ uint32_t h[kHistBins];
+    __shared__ uint32_t scan[kThreads];
+    __shared__ uint32_t found[2];
     const uint32_t l = blockIdx.x, tid = threadIdx.x;
     const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
+    if (A.topk) {
+        // level-1 digit (bits 30..20) of the layer's k-th largest |S|; the histogram is cleared for the next
+        // step.  These are scratch results: harmless when the step turns out to be skipped.
+        uint32_t *gh = A.hist + (uint64_t)l * kHistBins;
+        for (int b = tid; b < kHistBins; b += kThreads) { h[b] = gh[b]; gh[b] = 0u; }
+        __syncthreads();
+        const uint32_t k = (uint32_t)A.seg_k[l];
+        block_find_bin<true>(h, kHistBins, k, scan, found);
+        if (tid == 0) {
+            SelectState s;
+            s.prefix = found[0];
+            s.remaining = k - found[1];
+            s.thr_bits = 0u; s.take_equal = 0u; s.surplus = 0u; s.pad = 0u;
+            A.sel[l] = s;
+            A.cand_count[l] = 0u;
+        }
+    }
     double s1 = 0.0, s2 = 0.0, sa = 0.0, bad = 0.0;
     uint32_t amax = 0u, amin = 0xFFFFFFFFu;
     for (uint32_t i = lo + tid; i < hi; i += kThreads) {
@@ -661,83 +721,12 @@ __global__ void __launch_bounds__(kThreads) k_probe(float *z, uint64_t n_vec, ui
 // ------------------------------------------------------------------ top-k: radix select on |S| bit patterns
 //
 // |S| >= 0, so the order of the values is the order of their 31-bit patterns.  Level 1 (bits 30..20)
-// is counted during the sweep.  k_select1 finds, per layer, the bin b1 that holds the k-th largest
+// is counted during the sweep.  k_decide finds, per layer, the bin b1 that holds the k-th largest
 // value.  One more pass over |S| (k_mask_compact) sets the mask bits of every element in a bin above
 // b1 and appends the elements of bin b1 (value, index in layer) to the layer's candidate list.
 // k_resolve then finishes the selection on the candidates alone: two more value digits and, if more
 // candidates equal the threshold than are to be taken, three digits of the index (lower index first).
 // The result does not depend on the order in which candidates were appended.
-
-constexpr int kScanChunk = kHistBins / kThreads;
-
-// Whole block: the bin in which the `need`-th element falls when bins are walked from the top
-// (DESC) or from the bottom, and how many elements lie in the bins walked before it.
-template <bool DESC>
-__device__ __forceinline__ void block_find_bin(const uint32_t *h, int bins, uint32_t need, uint32_t *scan /*[kThreads]*/,
-                                               uint32_t *out /*[2]*/)
-{
-    const int tid = threadIdx.x, per = bins / kThreads;
-    uint32_t mine = 0;
-    for (int j = 0; j < per; ++j) {
-        const int pos = per * tid + j;
-        mine += h[DESC ? bins - 1 - pos : pos];
-    }
-    scan[tid] = mine;
-    __syncthreads();
-    for (int o = 1; o < kThreads; o <<= 1) {
-        const uint32_t add = tid >= o ? scan[tid - o] : 0u;
-        __syncthreads();
-        scan[tid] += add;
-        __syncthreads();
-    }
-    const uint32_t incl = scan[tid], before_me = incl - mine;
-    if (before_me < need && need <= incl) {
-        uint32_t cum = before_me;
-        for (int j = 0; j < per; ++j) {
-            const int pos = per * tid + j;
-            const int b = DESC ? bins - 1 - pos : pos;
-            const uint32_t cnt = h[b];
-            if (cum < need && need <= cum + cnt) { out[0] = (uint32_t)b; out[1] = cum; }
-            cum += cnt;
-        }
-    }
-    __syncthreads();
-}
-
-struct SelectArgs {
-    uint32_t *hist;              // [L][kHistBins]
-    SelectState *sel;            // [L]
-    uint32_t *cand_count;        // [L]
-    uint32_t *mask;
-    const uint64_t *seg_off, *seg_len, *seg_k;
-    const Status *status;
-};
-
-// One block per layer: level-1 bin of the k-th largest |S|; clears the histogram for the next step,
-// the candidate counter, and the (at most two) mask words the layer shares with a neighbour or a gap.
-__global__ void __launch_bounds__(kThreads) k_select1(const SelectArgs A)
-{
-    __shared__ uint32_t h[kHistBins];
-    __shared__ uint32_t scan[kThreads];
-    __shared__ uint32_t found[2];
-    const uint32_t l = blockIdx.x, tid = threadIdx.x;
-    uint32_t *gh = A.hist + (uint64_t)l * kHistBins;
-    for (int b = tid; b < kHistBins; b += kThreads) { h[b] = gh[b]; gh[b] = 0u; }
-    if (A.status->skipped) return;
-    __syncthreads();
-    block_find_bin<true>(h, kHistBins, (uint32_t)A.seg_k[l], scan, found);
-    if (tid == 0) {
-        SelectState s;
-        s.prefix = found[0];
-        s.remaining = (uint32_t)A.seg_k[l] - found[1];
-        s.thr_bits = 0u; s.take_equal = 0u; s.surplus = 0u; s.pad = 0u;
-        A.sel[l] = s;
-        A.cand_count[l] = 0u;
-        const uint64_t b = A.seg_off[l], e = b + A.seg_len[l];
-        if (b & 31u) A.mask[b >> 5] = 0u;
-        if (e & 31u) A.mask[e >> 5] = 0u;
-    }
-}
 
 struct MaskArgs {
     const Item *items;
@@ -763,7 +752,7 @@ __global__ void __launch_bounds__(kThreads) k_mask_compact(const MaskArgs A)
         const Item item = A.items[it];
         if (item.len == 0u) { if (lane == 0) A.p_mass[it] = 0.0; continue; }
         const uint64_t begin = item.begin, end = begin + item.len;
-        const uint64_t seg_b = A.seg_off[item.seg], seg_e = seg_b + A.seg_len[item.seg];
+        const uint64_t seg_b = A.seg_off[item.seg];
         const uint32_t b1 = A.sel[item.seg].prefix;
         uint32_t *cval = A.cand_val + seg_b, *cidx = A.cand_idx + seg_b;
         double mass = 0.0;
@@ -807,15 +796,15 @@ __global__ void __launch_bounds__(kThreads) k_mask_compact(const MaskArgs A)
                     if (ok[e] && bin == b1) cand |= 1u << e;
                 }
                 // candidates: one slot reservation per warp and row
-                const uint32_t n_mine = (uint32_t)__popc(cand);
-                uint32_t incl = n_mine;
+                if (__any_sync(0xFFFFFFFFu, cand != 0u)) {
+                    const uint32_t n_mine = (uint32_t)__popc(cand);
+                    uint32_t incl = n_mine;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                    if ((int)lane >= o) incl += t;
-                }
-                const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                if (total) {
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                        if ((int)lane >= o) incl += t;
+                    }
+                    const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
                     uint32_t base = 0;
                     if (lane == 31) base = atomicAdd(A.cand_count + item.seg, total);
                     base = __shfl_sync(0xFFFFFFFFu, base, 31) + incl - n_mine;
@@ -835,7 +824,11 @@ __global__ void __launch_bounds__(kThreads) k_mask_compact(const MaskArgs A)
                         *dst = word;                          // the word lies entirely inside this item
                     } else if (w0 + 32u > begin && w0 < end) {
                         // cut by the layer's first or last element (items are cut on multiples of 128 inside a
-                        // layer): the word is shared with a neighbour or a gap and was cleared by k_select1
+                        // layer): the other bits of this word belong to a neighbour or a gap, so replace only ours
+                        const uint32_t lo_bit = begin > w0 ? (uint32_t)(begin - w0) : 0u;
+                        const uint32_t hi_bit = end < w0 + 32u ? (uint32_t)(end - w0) : 32u;     // exclusive
+                        const uint32_t ours = (hi_bit == 32u ? 0xFFFFFFFFu : ((1u << hi_bit) - 1u)) & ~((1u << lo_bit) - 1u);
+                        atomicAnd(dst, ~ours);
                         if (word) atomicOr(dst, word);
                     }
                 }
@@ -879,14 +872,26 @@ __global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
 
     // value digits: bits 19..9, then bits 8..0
     clear(kHistBins);
-    for (uint32_t j = tid; j < m; j += kThreads) atomicAdd(&h[(cv[j] >> 9) & 2047u], 1u);
+    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * 8) {
+        uint32_t v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { const uint32_t j = j0 + u * kThreads + tid; v[u] = j < m ? __ldg(cv + j) : 0xFFFFFFFFu; }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) if (v[u] != 0xFFFFFFFFu) atomicAdd(&h[(v[u] >> 9) & 2047u], 1u);
+    }
     __syncthreads();
     block_find_bin<true>(h, kHistBins, s.remaining, scan, found);
     const uint32_t b2 = found[0], r2 = s.remaining - found[1];
     const uint32_t pre22 = (b1 << 11) | b2;
     __syncthreads();
     clear(512);
-    for (uint32_t j = tid; j < m; j += kThreads) { const uint32_t v = cv[j]; if ((v >> 9) == pre22) atomicAdd(&h[v & 511u], 1u); }
+    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * 8) {
+        uint32_t v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { const uint32_t j = j0 + u * kThreads + tid; v[u] = j < m ? __ldg(cv + j) : 0xFFFFFFFFu; }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) if ((v[u] >> 9) == pre22) atomicAdd(&h[v[u] & 511u], 1u);
+    }
     __syncthreads();
     block_find_bin<true>(h, 512, r2, scan, found);
     const uint32_t thr = (pre22 << 9) | found[0];
@@ -921,13 +926,23 @@ __global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
     // set the bits of the taken candidates; their sum is exact: all share sign and exponent
     // (the exponent is part of the level-1 digit), so it is count * 2^e + (sum of mantissas) * 2^(e-23)
     unsigned long long cnt = 0ull, mant = 0ull;
-    for (uint32_t j = tid; j < m; j += kThreads) {
-        const uint32_t v = cv[j], ix = ci[j];
-        if (v > thr || (v == thr && ix <= idx_limit)) {
-            const uint64_t i = off + ix;
-            atomicOr(A.mask + (i >> 5), 1u << (i & 31u));
-            ++cnt;
-            mant += v & 0x007FFFFFu;
+    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * 8) {
+        uint32_t v[8], ix[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t j = j0 + u * kThreads + tid;
+            v[u] = j < m ? __ldg(cv + j) : 0u;          // 0 is never taken: thr > 0 here or handled by the index rule
+            ix[u] = j < m ? __ldg(ci + j) : 0xFFFFFFFFu;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t j = j0 + u * kThreads + tid;
+            if (j < m && (v[u] > thr || (v[u] == thr && ix[u] <= idx_limit))) {
+                const uint64_t i = off + ix[u];
+                atomicOr(A.mask + (i >> 5), 1u << (i & 31u));
+                ++cnt;
+                mant += v[u] & 0x007FFFFFu;
+            }
         }
     }
     if (tid < 2) acc_u64[tid] = 0ull;

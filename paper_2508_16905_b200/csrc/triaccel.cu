@@ -421,20 +421,19 @@ int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
     da.hp = hyper_of(h->hp); da.eta0 = h->hp.eta0; da.L = h->L;
     da.has_hz = Hz ? 1u : 0u; da.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; da.topk = topk ? 1u : 0u;
     da.step = step;
+    da.hist = d.hist; da.sel = d.sel; da.cand_count = d.cand_count; da.seg_k = d.seg_k;
     ta::k_decide<<<h->L, ta::kThreads, 0, s>>>(da);
     ++h->launches;
 
     if (topk) {
         const int grid = grid_for(h);
-        ta::SelectArgs se{d.hist, d.sel, d.cand_count, d.mask, d.seg_off, d.seg_len, d.seg_k, d.status};
-        ta::k_select1<<<h->L, ta::kThreads, 0, s>>>(se);
         ta::MaskArgs ma{d.items, h->n_items, h->n_batches, d.abs_s, d.mask, d.p_mass, d.sel, d.seg_off, d.seg_len,
                         d.cand_count, d.cand_val, d.cand_idx, d.status};
         ta::k_mask_compact<<<grid, ta::kThreads, 0, s>>>(ma);
         ta::ResolveArgs ra{d.item_lo, d.seg_off, d.seg_len, d.cand_count, d.cand_val, d.cand_idx, d.mask, d.p_mass,
                            d.scratch, d.sel, d.state, d.status};
         ta::k_resolve<<<h->L, ta::kThreads, 0, s>>>(ra);
-        h->launches += 3;
+        h->launches += 2;
     }
 
     if (timed) cudaEventRecord(ev[2], s);
