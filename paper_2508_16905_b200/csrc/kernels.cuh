@@ -536,7 +536,11 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
         // level-1 digit (bits 30..20) of the layer's k-th largest |S|; the histogram is cleared for the next
         // step.  These are scratch results: harmless when the step turns out to be skipped.
         uint32_t *gh = A.hist + (uint64_t)l * kHistBins;
-        for (int b = tid; b < kHistBins; b += kThreads) { h[b] = gh[b]; gh[b] = 0u; }
+        uint32_t bins[kHistBins / kThreads];
+#pragma unroll
+        for (int j = 0; j < kHistBins / kThreads; ++j) bins[j] = gh[j * kThreads + tid];      // all loads in flight at once
+#pragma unroll
+        for (int j = 0; j < kHistBins / kThreads; ++j) { h[j * kThreads + tid] = bins[j]; gh[j * kThreads + tid] = 0u; }
         __syncthreads();
         const uint32_t k = (uint32_t)A.seg_k[l];
         block_find_bin<true>(h, kHistBins, k, scan, found);
@@ -742,9 +746,43 @@ struct MaskArgs {
     const Status *status;
 };
 
+constexpr uint32_t kStageCap = 384;      // candidates a warp collects in shared memory before it reserves list slots
+
+// Stages this lane's candidates (bit e of `cand` = element e of its vector) in the warp's shared-memory
+// buffer, behind the `running` ones already there.  Whole warp; `running` stays warp-uniform.
+__device__ __forceinline__ void stage_candidates(uint32_t cand, const uint32_t (&ab)[4], uint32_t local0, uint32_t lane,
+                                                 uint32_t &running, uint32_t *sval, uint32_t *sidx)
+{
+    if (!__any_sync(0xFFFFFFFFu, cand != 0u)) return;
+    const uint32_t n_mine = (uint32_t)__popc(cand);
+    uint32_t incl = n_mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if ((int)lane >= o) incl += t;
+    }
+    uint32_t base = running + incl - n_mine;
+    running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+#pragma unroll
+    for (uint32_t e = 0; e < 4; ++e)
+        if (cand & (1u << e)) { sval[base] = ab[e]; sidx[base] = local0 + e; ++base; }
+}
+
+// 8 lanes make one 32-bit mask word out of their 4-bit pieces.
+__device__ __forceinline__ uint32_t gather_word(uint32_t nib, uint32_t lane)
+{
+    uint32_t word = nib << ((lane & 7u) * 4u);
+    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+    return word;
+}
+
 __global__ void __launch_bounds__(kThreads) k_mask_compact(const MaskArgs A)
 {
     if (A.status->skipped) return;
+    __shared__ uint32_t sh_val[kWarps][kStageCap];
+    __shared__ uint32_t sh_idx[kWarps][kStageCap];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
         const uint32_t it = batch * kWarps + warp;
@@ -754,87 +792,96 @@ __global__ void __launch_bounds__(kThreads) k_mask_compact(const MaskArgs A)
         const uint64_t begin = item.begin, end = begin + item.len;
         const uint64_t seg_b = A.seg_off[item.seg];
         const uint32_t b1 = A.sel[item.seg].prefix;
-        uint32_t *cval = A.cand_val + seg_b, *cidx = A.cand_idx + seg_b;
+        uint32_t *sval = sh_val[warp], *sidx = sh_idx[warp];
+        uint32_t staged = 0u;
         double mass = 0.0;
+        // moves the staged candidates to the layer's list: one slot reservation for all of them
+        auto flush = [&]() {
+            if (staged == 0u) return;
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(A.cand_count + item.seg, staged);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            __syncwarp();
+            for (uint32_t j = lane; j < staged; j += 32) {
+                A.cand_val[seg_b + base + j] = sval[j];
+                A.cand_idx[seg_b + base + j] = sidx[j];
+            }
+            __syncwarp();
+            staged = 0u;
+        };
+
+        // a row that is cut by the first or last element of the layer
+        auto partial_row = [&](uint64_t row) {
+            const uint64_t i0 = row * 128ull + lane * 4u;
+            uint32_t ab[4] = {0u, 0u, 0u, 0u};
+            uint32_t nib = 0u, cand = 0u;
+            for (uint32_t e = 0; e < 4; ++e) {
+                if (i0 + e >= begin && i0 + e < end) {
+                    ab[e] = __float_as_uint(A.abs_s[i0 + e]);
+                    const uint32_t bin = ab[e] >> 20;
+                    if (bin > b1) { nib |= 1u << e; mass += (double)__uint_as_float(ab[e]); }
+                    if (bin == b1) cand |= 1u << e;
+                }
+            }
+            if (staged + 128u > kStageCap) flush();
+            stage_candidates(cand, ab, (uint32_t)(i0 - seg_b), lane, staged, sval, sidx);
+            const uint32_t word = gather_word(nib, lane);
+            if ((lane & 7u) == 0u) {
+                const uint64_t w0 = row * 128ull + (lane >> 3) * 32ull;     // first element of this word
+                uint32_t *dst = A.mask + (w0 >> 5);
+                if (w0 >= begin && w0 + 32u <= end) {
+                    *dst = word;
+                } else if (w0 + 32u > begin && w0 < end) {
+                    // the other bits of this word belong to a neighbouring layer or a gap: replace only ours
+                    const uint32_t lo_bit = begin > w0 ? (uint32_t)(begin - w0) : 0u;
+                    const uint32_t hi_bit = end < w0 + 32u ? (uint32_t)(end - w0) : 32u;     // exclusive
+                    const uint32_t ours = (hi_bit == 32u ? 0xFFFFFFFFu : ((1u << hi_bit) - 1u)) & ~((1u << lo_bit) - 1u);
+                    atomicAnd(dst, ~ours);
+                    if (word) atomicOr(dst, word);
+                }
+            }
+        };
+        // a row entirely inside the item: its four mask words are owned by this warp
+        auto full_row = [&](uint64_t row, const float4 v) {
+            const uint32_t ab[4] = {__float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z), __float_as_uint(v.w)};
+            uint32_t nib = 0u, cand = 0u;
+            float above = 0.f;
+#pragma unroll
+            for (uint32_t e = 0; e < 4; ++e) {
+                const uint32_t bin = ab[e] >> 20;
+                if (bin > b1) { nib |= 1u << e; above += __uint_as_float(ab[e]); }
+                if (bin == b1) cand |= 1u << e;
+            }
+            mass += (double)above;
+            if (staged + 128u > kStageCap) flush();
+            stage_candidates(cand, ab, (uint32_t)(row * 128ull - seg_b) + lane * 4u, lane, staged, sval, sidx);
+            const uint32_t word = gather_word(nib, lane);
+            if ((lane & 7u) == 0u) A.mask[row * 4ull + (lane >> 3)] = word;
+        };
+
         const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
-        constexpr int U = 4;
-        uint64_t row = row_first;
-        while (row <= row_last) {
-            const bool group_full = row * 128ull >= begin && (row + U) * 128ull <= end;
-            const int rows = group_full ? U : 1;
-            float4 v[U];
-            bool full = group_full;
-            if (group_full) {
+        const uint64_t full_lo = (begin + 127) >> 7, full_hi = end >> 7;
+        const bool head_partial = (begin & 127u) != 0u;
+        const bool tail_partial = (end & 127u) != 0u && !(head_partial && row_last == row_first);
+        if (head_partial) partial_row(row_first);
+        if (full_hi > full_lo) {
+            constexpr int U = 8;
+            uint64_t row = full_lo;
+            while (row + U <= full_hi) {
+                float4 v[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) v[u] = __ldcs(reinterpret_cast<const float4 *>(A.abs_s + (row + u) * 128ull + lane * 4u));
-            } else {
-                full = row * 128ull >= begin && row * 128ull + 128u <= end;
-                if (full) v[0] = __ldcs(reinterpret_cast<const float4 *>(A.abs_s + row * 128ull + lane * 4u));
+#pragma unroll
+                for (int u = 0; u < U; ++u) full_row(row + u, v[u]);
+                row += U;
             }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (u >= rows) break;
-                const uint64_t i0 = (row + u) * 128ull + lane * 4u;
-                uint32_t ab[4];
-                bool ok[4];
-                if (full) {
-                    ab[0] = __float_as_uint(v[u].x); ab[1] = __float_as_uint(v[u].y);
-                    ab[2] = __float_as_uint(v[u].z); ab[3] = __float_as_uint(v[u].w);
-                    ok[0] = ok[1] = ok[2] = ok[3] = true;
-                } else {
-#pragma unroll
-                    for (uint32_t e = 0; e < 4; ++e) {
-                        ok[e] = i0 + e >= begin && i0 + e < end;
-                        ab[e] = ok[e] ? __float_as_uint(A.abs_s[i0 + e]) : 0u;
-                    }
-                }
-                uint32_t nib = 0u, cand = 0u;
-#pragma unroll
-                for (uint32_t e = 0; e < 4; ++e) {
-                    const uint32_t bin = ab[e] >> 20;
-                    if (ok[e] && bin > b1) { nib |= 1u << e; mass += (double)__uint_as_float(ab[e]); }
-                    if (ok[e] && bin == b1) cand |= 1u << e;
-                }
-                // candidates: one slot reservation per warp and row
-                if (__any_sync(0xFFFFFFFFu, cand != 0u)) {
-                    const uint32_t n_mine = (uint32_t)__popc(cand);
-                    uint32_t incl = n_mine;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                        if ((int)lane >= o) incl += t;
-                    }
-                    const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                    uint32_t base = 0;
-                    if (lane == 31) base = atomicAdd(A.cand_count + item.seg, total);
-                    base = __shfl_sync(0xFFFFFFFFu, base, 31) + incl - n_mine;
-#pragma unroll
-                    for (uint32_t e = 0; e < 4; ++e)
-                        if (cand & (1u << e)) { cval[base] = ab[e]; cidx[base] = (uint32_t)(i0 + e - seg_b); ++base; }
-                }
-                // mask words: 8 lanes make one 32-bit word
-                uint32_t word = nib << ((lane & 7u) * 4u);
-                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
-                word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
-                if ((lane & 7u) == 0u) {
-                    const uint64_t w0 = (row + u) * 128ull + (lane >> 3) * 32ull;     // first element of this word
-                    uint32_t *dst = A.mask + (w0 >> 5);
-                    if (w0 >= begin && w0 + 32u <= end) {
-                        *dst = word;                          // the word lies entirely inside this item
-                    } else if (w0 + 32u > begin && w0 < end) {
-                        // cut by the layer's first or last element (items are cut on multiples of 128 inside a
-                        // layer): the other bits of this word belong to a neighbour or a gap, so replace only ours
-                        const uint32_t lo_bit = begin > w0 ? (uint32_t)(begin - w0) : 0u;
-                        const uint32_t hi_bit = end < w0 + 32u ? (uint32_t)(end - w0) : 32u;     // exclusive
-                        const uint32_t ours = (hi_bit == 32u ? 0xFFFFFFFFu : ((1u << hi_bit) - 1u)) & ~((1u << lo_bit) - 1u);
-                        atomicAnd(dst, ~ours);
-                        if (word) atomicOr(dst, word);
-                    }
-                }
+            while (row < full_hi) {
+                full_row(row, __ldcs(reinterpret_cast<const float4 *>(A.abs_s + row * 128ull + lane * 4u)));
+                ++row;
             }
-            row += rows;
         }
+        if (tail_partial) partial_row(row_last);
+        flush();
         mass = warp_sum(mass);
         if (lane == 0) A.p_mass[it] = mass;
     }
@@ -863,12 +910,13 @@ __global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
     __shared__ unsigned long long acc_u64[2];
     const uint32_t l = blockIdx.x, tid = threadIdx.x;
     const uint64_t off = A.seg_off[l];
-    const uint32_t m = A.cand_count[l];
-    const uint32_t *cv = A.cand_val + off, *ci = A.cand_idx + off;
     SelectState s = A.sel[l];
     const uint32_t b1 = s.prefix;
 
     auto clear = [&](int bins) { for (int b = tid; b < bins; b += kThreads) h[b] = 0u; __syncthreads(); };
+
+    const uint32_t m = A.cand_count[l];
+    const uint32_t *cv = A.cand_val + off, *ci = A.cand_idx + off;
 
     // value digits: bits 19..9, then bits 8..0
     clear(kHistBins);
