@@ -47,7 +47,8 @@ struct LayerScratch {
 struct Status {
     unsigned long long step, nonfinite;
     uint32_t skipped, near_count;
-    uint32_t done_counter, pad;
+    uint32_t done_counter, device_error;   // device_error: a bounded wait inside a kernel ran out
+    uint32_t near_stage, pad;              // near-threshold layers of a step that may still be skipped
 };
 
 // Per-layer bookkeeping of the radix select.
@@ -237,15 +238,14 @@ template <int P, bool TOPK> struct SweepAcc {
     }
 };
 
+// One batch (eight items, one per warp) of the sweep.  Called by the whole block.
 template <int P, bool BF16, bool TOPK>
-__global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
+__device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, uint32_t *sh_hist)
 {
     constexpr int PP = P > 0 ? P : 1;
     constexpr int U = (P <= 1) ? 8 : (P == 2 ? 4 : 2);     // rows in flight per lane
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
-
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+    {
         const uint32_t it = batch * kWarps + warp;
         // a batch whose items share one layer counts its histogram in shared memory and flushes it once
         bool uniform = false;
@@ -419,6 +419,13 @@ __global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
     }
 }
 
+template <int P, bool BF16, bool TOPK>
+__global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
+{
+    __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK>(A, batch, sh_hist);
+}
+
 // ------------------------------------------------------------------ decisions
 
 // Whole block: the bin in which the `need`-th element falls when bins are walked from the top
@@ -489,34 +496,47 @@ __device__ __forceinline__ LayerScratch load_scratch(const LayerScratch *p)
     return sc;
 }
 
-// Sec. 3.1 (EMAs, code cases), Sec. 3.2 (step size, promotion), Sec. 3.4 (control interval).
-__device__ __forceinline__ uint32_t commit_layer(const DecideArgs &A, uint32_t l)
+struct DecideParams {
+    Hyper hp;
+    float eta0;
+    uint32_t has_hz, control, topk;
+};
+
+// Sec. 3.1 (EMAs, code cases), Sec. 3.2 (step size, promotion), Sec. 3.4 (control interval):
+// the new state of one layer from its old state and this step's statistics.
+__device__ __forceinline__ LayerState decide_layer(const DecideParams &P, LayerState st, const LayerScratch &sc, uint32_t &near)
 {
-    LayerState st = A.state[l];
-    const LayerScratch sc = load_scratch(A.scratch + l);
-    const double beta = (double)A.hp.beta;
+    const double beta = (double)P.hp.beta;
     st.grad_mean = sc.mean;
     st.grad_var = sc.var;
     st.ema_mean = (float)(beta * (double)st.ema_mean + (1.0 - beta) * sc.mean);
     st.ema_var = (float)(beta * (double)st.ema_var + (1.0 - beta) * sc.var);
-    if (A.has_hz) {
-        st.lambda_max = __fdiv_rn(__uint_as_float(sc.amax), (float)A.hp.num_probes);
-        if (!A.topk) { st.thr = __uint_as_float(sc.amin); st.topk_mass = 1.0; }
+    if (P.has_hz) {
+        st.lambda_max = __fdiv_rn(__uint_as_float(sc.amax), (float)P.hp.num_probes);
+        if (!P.topk) { st.thr = __uint_as_float(sc.amin); st.topk_mass = 1.0; }
     }
-    uint32_t near = 0;
-    if (A.control) {
+    near = 0;
+    if (P.control) {
         const float v = st.ema_var;
-        uint32_t code = v < A.hp.tau_low ? 0u : (v < A.hp.tau_high ? 1u : 2u);
-        if (st.lambda_max > A.hp.tau_curv && code < 2u) code += 1u;
+        uint32_t code = v < P.hp.tau_low ? 0u : (v < P.hp.tau_high ? 1u : 2u);
+        if (st.lambda_max > P.hp.tau_curv && code < 2u) code += 1u;
         st.code = code;
-        st.eta_scale = __fdiv_rn(1.0f, __fadd_rn(1.0f, __fmul_rn(A.hp.alpha, st.lambda_max)));
-        if (fabs((double)v - (double)A.hp.tau_low) <= 1e-5 * fabs((double)A.hp.tau_low)) near = 1;
-        if (fabs((double)v - (double)A.hp.tau_high) <= 1e-5 * fabs((double)A.hp.tau_high)) near = 1;
-        if (fabs((double)st.lambda_max - (double)A.hp.tau_curv) <= 1e-5 * fabs((double)A.hp.tau_curv)) near = 1;
+        st.eta_scale = __fdiv_rn(1.0f, __fadd_rn(1.0f, __fmul_rn(P.hp.alpha, st.lambda_max)));
+        if (fabs((double)v - (double)P.hp.tau_low) <= 1e-5 * fabs((double)P.hp.tau_low)) near = 1;
+        if (fabs((double)v - (double)P.hp.tau_high) <= 1e-5 * fabs((double)P.hp.tau_high)) near = 1;
+        if (fabs((double)st.lambda_max - (double)P.hp.tau_curv) <= 1e-5 * fabs((double)P.hp.tau_curv)) near = 1;
         st.near = near;
     }
-    st.eta = __fmul_rn(A.eta0, st.eta_scale);
-    A.state[l] = st;
+    st.eta = __fmul_rn(P.eta0, st.eta_scale);
+    return st;
+}
+
+__device__ __forceinline__ uint32_t commit_layer(const DecideArgs &A, uint32_t l)
+{
+    DecideParams P;
+    P.hp = A.hp; P.eta0 = A.eta0; P.has_hz = A.has_hz; P.control = A.control; P.topk = A.topk;
+    uint32_t near;
+    A.state[l] = decide_layer(P, A.state[l], load_scratch(A.scratch + l), near);
     return near;
 }
 
@@ -626,20 +646,22 @@ __device__ __forceinline__ uint16_t cast16(float x, uint32_t code)
 }
 
 // w <- fl32(w - eta_l g) (Sec. 3.2, Sec. 4.1); c <- RNE cast of the new w for FP16 / BF16 layers (Sec. 2).
-template <bool BF16>
-__global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
+// One batch of the update.  `decision(seg, eta, code)` supplies the layer's step size and precision code.
+template <bool BF16, typename Decision>
+__device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, const Decision &decision)
 {
-    if (A.status->skipped) return;
     constexpr int U = 4;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+    {
         const uint32_t it = batch * kWarps + warp;
-        if (it >= A.n_items) continue;
+        if (it >= A.n_items) return;
         const Item item = A.items[it];
-        if (item.len == 0u) continue;
+        if (item.len == 0u) return;
         const uint64_t begin = item.begin, end = begin + item.len;
-        const float neg_eta = -A.state[item.seg].eta;
-        const uint32_t code = A.state[item.seg].code;
+        float eta;
+        uint32_t code;
+        decision(item.seg, eta, code);
+        const float neg_eta = -eta;
 
         auto partial_row = [&](uint64_t row) {
             const uint64_t i0 = row * 128ull + lane * 4u;
@@ -700,6 +722,184 @@ __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
         }
         if (tail_partial) partial_row(row_last);
     }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
+{
+    if (A.status->skipped) return;
+    const LayerState *state = A.state;
+    auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) apply_batch<BF16>(A, batch, decision);
+}
+
+// ------------------------------------------------------------------ one launch for small models
+//
+// When the whole model is small, three launches cost more than the data movement.  k_fused runs the
+// sweep, the decisions and the update in ONE cooperative launch (every block resident), separated by
+// two grid-wide barriers.  The gradient (and the weights, prefetched during the sweep) is then still
+// in L2 when the update reads it.  Waits are bounded: a block that gives up sets status->device_error
+// and returns, so a lost block cannot hang the GPU.
+
+// What the block that owns a layer publishes for all blocks between the two barriers.
+struct LayerVerdict {
+    float eta;           // step size of the layer if the step is committed
+    uint32_t code_bad;   // precision code in the low byte; bit 31: the layer saw a non-finite input
+};
+
+struct FusedArgs {
+    SweepArgs sweep;
+    ApplyArgs apply;
+    const uint32_t *item_lo;
+    const uint64_t *seg_len;
+    LayerVerdict *verdict;          // [L]
+    LayerState *state;              // [L]
+    Status *status;
+    DecideParams dp;
+    uint32_t L;
+    unsigned long long step;
+    unsigned long long *barrier;    // arrivals, only ever incremented
+    unsigned long long barrier_base;// arrivals before this launch
+    uint32_t prefetch_w;
+};
+
+constexpr uint32_t kBarrierSpinLimit = 1u << 22;     // with a 64 ns back-off: gives up after roughly a second
+
+// Grid-wide barrier on a monotonic arrival counter.  Returns false when the wait ran out.
+__device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsigned long long target, Status *status)
+{
+    __shared__ uint32_t ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1ull);
+        uint32_t spins = 0;
+        bool arrived = true;
+        while (*reinterpret_cast<volatile unsigned long long *>(counter) < target) {
+            if (++spins > kBarrierSpinLimit) { arrived = false; break; }
+            __nanosleep(64);
+        }
+        if (!arrived) atomicExch(&status->device_error, 1u);
+        __threadfence();
+        ok = arrived ? 1u : 0u;
+    }
+    __syncthreads();
+    return ok != 0u;
+}
+
+template <int P, bool BF16>
+__global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
+{
+    extern __shared__ unsigned char dyn_smem[];
+    float *sh_eta = reinterpret_cast<float *>(dyn_smem);                 // [L]
+    uint32_t *sh_code = reinterpret_cast<uint32_t *>(dyn_smem) + A.L;    // [L]
+    __shared__ double red[kWarps];
+    __shared__ uint32_t red_u[2][kWarps];
+    const uint32_t tid = threadIdx.x;
+    const unsigned long long G = gridDim.x;
+
+    // phase 1: sweep
+    if (blockIdx.x == 0 && tid == 0) A.status->near_stage = 0u;
+    for (uint32_t batch = blockIdx.x; batch < A.sweep.n_batches; batch += gridDim.x)
+        sweep_batch<P, BF16, false>(A.sweep, batch, nullptr);
+    if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) return;
+
+    // DRAM is idle until the update starts: pull this block's weights into L2 meanwhile
+    if (A.prefetch_w) {
+        for (uint32_t batch = blockIdx.x; batch < A.sweep.n_batches; batch += gridDim.x) {
+            const uint32_t it = batch * kWarps + (tid >> 5);
+            if (it < A.sweep.n_items) {
+                const Item item = A.sweep.items[it];
+                const char *base = reinterpret_cast<const char *>(A.apply.w + item.begin);
+                for (uint32_t off = (tid & 31u) * 128u; off < item.len * 4u; off += 32u * 128u)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+            }
+        }
+    }
+
+    // phase 2: blocks share the layers.  The owner of a layer combines the layer's item partials in a fixed
+    // order, takes the layer's decisions, keeps the new state in registers and publishes step size, code and
+    // its non-finite flag for everybody.  At most kOwned layers per block.
+    constexpr int kOwned = 4;
+    LayerState mine[kOwned];
+    uint32_t n_owned = 0;
+    for (uint32_t l = blockIdx.x; l < A.L; l += gridDim.x) {
+        const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
+        for (uint32_t i = lo + tid; i < hi; i += kThreads) {
+            s1 += __ldcg(A.sweep.p_s1 + i);
+            s2 += __ldcg(A.sweep.p_s2 + i);
+            bad |= __ldcg(A.sweep.p_bad + i);
+            if (P > 0) {
+                amax = max(amax, __ldcg(A.sweep.p_amax + i));
+                amin = min(amin, __ldcg(A.sweep.p_amin + i));
+            }
+        }
+        s1 = block_sum(s1, red);
+        s2 = block_sum(s2, red);
+        amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+        amin = __reduce_min_sync(0xFFFFFFFFu, amin);
+        bad = (uint32_t)__syncthreads_or((int)bad);
+        if ((tid & 31) == 0) { red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
+            const double n = (double)A.seg_len[l];
+            const double mu = s1 / n;
+            double var = s2 / n - mu * mu;
+            if (!(var > 0.0)) var = 0.0;
+            LayerScratch sc;
+            sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = bad; sc.amax = amax; sc.amin = amin;
+            uint32_t near;
+            const LayerState st = decide_layer(A.dp, A.state[l], sc, near);
+            if (n_owned < (uint32_t)kOwned) mine[n_owned] = st;
+            LayerVerdict v;
+            v.eta = st.eta;
+            v.code_bad = st.code | (bad ? 0x80000000u : 0u);
+            A.verdict[l] = v;
+            if (near) atomicAdd(&A.status->near_stage, 1u);
+        }
+        ++n_owned;
+    }
+    if (!grid_barrier(A.barrier, A.barrier_base + 2ull * G, A.status)) return;
+
+    // every block reads all verdicts: is the step committed, and with which step sizes and codes
+    uint32_t any_bad = 0u;
+    for (uint32_t l = tid; l < A.L; l += kThreads) {
+        const float eta = __ldcg(&A.verdict[l].eta);
+        const uint32_t cb = __ldcg(&A.verdict[l].code_bad);
+        sh_eta[l] = eta;
+        sh_code[l] = cb & 0xFFu;
+        any_bad |= cb >> 31;
+    }
+    any_bad = (uint32_t)__syncthreads_or((int)any_bad);      // also orders the shared-memory table before its use
+    if (blockIdx.x == 0 && tid == 0) {
+        A.status->step = A.step;
+        A.status->skipped = any_bad ? 1u : 0u;
+        if (!any_bad) {
+            A.status->nonfinite = 0ull;
+            if (A.dp.control) A.status->near_count = A.status->near_stage;
+        }
+    }
+    if (any_bad) {
+        // skipped step: nothing changes.  The exact count of non-finite values is summed by block 0.
+        if (blockIdx.x == 0) {
+            double total = 0.0;
+            for (uint32_t i = tid; i < A.sweep.n_items; i += kThreads) total += (double)__ldcg(A.sweep.p_bad + i);
+            total = block_sum(total, red);
+            if (tid == 0) A.status->nonfinite = (unsigned long long)total;
+        }
+        return;
+    }
+    if (tid == 0) {
+        uint32_t j = 0;
+        for (uint32_t l = blockIdx.x; l < A.L && j < (uint32_t)kOwned; l += gridDim.x, ++j) A.state[l] = mine[j];
+    }
+
+    // phase 3: update + cast
+    auto decision = [sh_eta, sh_code](uint32_t seg, float &eta, uint32_t &code) { eta = sh_eta[seg]; code = sh_code[seg]; };
+    for (uint32_t batch = blockIdx.x; batch < A.apply.n_batches; batch += gridDim.x) apply_batch<BF16>(A.apply, batch, decision);
 }
 
 // ------------------------------------------------------------------ probe writer

@@ -22,6 +22,8 @@ struct DeviceBuffers {
     ta::LayerState *state = nullptr;
     ta::LayerScratch *scratch = nullptr;
     ta::Status *status = nullptr;
+    ta::LayerVerdict *verdict = nullptr;          // fused launch: per-layer step size, code, non-finite flag
+    unsigned long long *barrier = nullptr;        // fused launch: grid-barrier arrivals
     double *p_s1 = nullptr, *p_s2 = nullptr, *p_sa = nullptr, *p_mass = nullptr;
     uint32_t *p_amax = nullptr, *p_amin = nullptr, *p_bad = nullptr;
     float *abs_s = nullptr;
@@ -55,6 +57,9 @@ struct ta_handle {
     std::vector<cudaEvent_t> events;      // 4 per timed step: before sweep, after sweep, after decisions, after update
     uint32_t timed_cap = 0, timed_used = 0;
     // top-k: the per-layer resolve kernel runs beside the update kernel on a stream of its own
+    bool fused_ok = false;                // small dense models: sweep + decisions + update in one cooperative launch
+    int fused_grid[2][5] = {};            // resident grid of each k_fused variant: [bf16][index of P in 0,1,2,4,8]
+    unsigned long long barrier_base = 0;  // barrier arrivals of all fused launches so far
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     DeviceBuffers d;
@@ -87,7 +92,7 @@ template <typename T> cudaError_t dev_alloc(T **p, size_t count)
 
 void free_all(DeviceBuffers &d)
 {
-    void *ptrs[] = {d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
+    void *ptrs[] = {d.verdict, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
                     d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
     for (void *p : ptrs)
@@ -148,6 +153,42 @@ template <bool BF16> bool dispatch_sweep(ta_handle *h, int P, const ta::SweepArg
     case 8: topk ? launch_sweep<8, BF16, true>(h, a, s) : launch_sweep<8, BF16, false>(h, a, s); return true;
     default: return false;
     }
+}
+
+int p_index(int P) { return P == 0 ? 0 : P == 1 ? 1 : P == 2 ? 2 : P == 4 ? 3 : 4; }
+
+template <int P, bool BF16> const void *fused_fn() { return reinterpret_cast<const void *>(&ta::k_fused<P, BF16>); }
+
+const void *fused_kernel(int P, bool bf16)
+{
+    switch (P) {
+    case 0: return bf16 ? fused_fn<0, true>() : fused_fn<0, false>();
+    case 1: return bf16 ? fused_fn<1, true>() : fused_fn<1, false>();
+    case 2: return bf16 ? fused_fn<2, true>() : fused_fn<2, false>();
+    case 4: return bf16 ? fused_fn<4, true>() : fused_fn<4, false>();
+    case 8: return bf16 ? fused_fn<8, true>() : fused_fn<8, false>();
+    default: return nullptr;
+    }
+}
+
+uint64_t fused_max_params()
+{
+    if (const char *env = getenv("TRIACCEL_FUSED_MAX_PARAMS")) return (uint64_t)atoll(env);
+    return 16ull << 20;
+}
+
+// A bounded wait inside a kernel ran out (a block of a cooperative launch never arrived): the step that
+// hit it is incomplete.  Reports it once and re-arms the barrier.
+int check_device_error(ta_handle *h)
+{
+    ta::Status s;
+    TA_CUDA(h, cudaMemcpy(&s, h->d.status, sizeof(s), cudaMemcpyDeviceToHost));
+    if (!s.device_error) return TA_OK;
+    s.device_error = 0u;
+    TA_CUDA(h, cudaMemcpy(h->d.status, &s, sizeof(s), cudaMemcpyHostToDevice));
+    if (h->d.barrier) TA_CUDA(h, cudaMemset(h->d.barrier, 0, sizeof(unsigned long long)));
+    h->barrier_base = 0;
+    return fail(h, TA_ERR_CUDA, "a bounded device-side wait ran out during the last step; its results are incomplete");
 }
 
 int default_mem_reader(void *, uint64_t *free_b, uint64_t *total_b)
@@ -235,8 +276,38 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     h->topk = hp->topk_ppm < 1000000u;
     h->mask_words = h->topk ? (n_total + 31) / 32 : 0;
 
+    // one-launch path for small dense models: needs a cooperative launch with every block resident
+    long long fused_blocks = 0;
+    {
+        int coop = 0;
+        TA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device));
+        const size_t smem = (size_t)L * 8;
+        if (coop && !h->topk && n_params <= fused_max_params() && smem <= 32 * 1024) {
+            const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
+            h->fused_ok = true;
+            fused_blocks = 1ll << 40;
+            for (int P : {0, (int)hp->num_probes}) {
+                int per_sm = 0;
+                TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(P, bf16), ta::kThreads, smem));
+                if (const char *env = getenv("TRIACCEL_FUSED_CTAS_PER_SM")) per_sm = std::min(per_sm, std::max(1, atoi(env)));
+                h->fused_grid[bf16][p_index(P)] = per_sm * h->sm_count;
+                fused_blocks = std::min<long long>(fused_blocks, (long long)per_sm * h->sm_count);
+                if (per_sm < 1 || (long long)per_sm * h->sm_count * 4 < (long long)L) h->fused_ok = false;
+            }
+        }
+    }
+
     // plan: items cut on a global grid of item_elems elements, clipped to each layer
     h->item_elems = choose_item_elems(n_params, h->sm_count);
+    if (h->fused_ok && !getenv("TRIACCEL_ITEM_ELEMS")) {
+        // one item per warp of the resident grid if the model is small enough: every phase is a single round
+        for (uint32_t cand = 512; cand <= 16384; cand += 512) {
+            unsigned long long count = 0;
+            for (uint32_t l = 0; l < L; ++l)
+                count += (table[l].offset + table[l].length - 1) / cand - table[l].offset / cand + 1;
+            if (count <= (unsigned long long)fused_blocks * ta::kWarps) { h->item_elems = cand; break; }
+        }
+    }
     std::vector<ta::Item> items;
     std::vector<uint32_t> item_lo(L + 1);
     std::vector<uint64_t> seg_off(L), seg_len(L);
@@ -264,6 +335,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     item_lo[L] = (uint32_t)items.size();
     h->n_items = (uint32_t)items.size();
     h->n_batches = (h->n_items + ta::kWarps - 1) / ta::kWarps;
+    if (h->fused_ok && std::min<long long>(fused_blocks, h->n_batches) * 4 < (long long)L) h->fused_ok = false;
     std::vector<uint32_t> batch_seg(h->n_batches, ta::kMixedBatch);
     for (uint32_t bt = 0; bt < h->n_batches; ++bt) {
         uint32_t seg = ta::kMixedBatch;
@@ -326,6 +398,11 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     TA_TRY(cudaMemcpy(d.state, init.data(), L * sizeof(ta::LayerState), cudaMemcpyHostToDevice));
     TA_TRY(cudaMemset(d.scratch, 0, L * sizeof(ta::LayerScratch)));
     TA_TRY(cudaMemset(d.status, 0, sizeof(ta::Status)));
+    if (h->fused_ok) {
+        TA_TRY(dev_alloc(&d.verdict, L));
+        TA_TRY(dev_alloc(&d.barrier, 1));
+        TA_TRY(cudaMemset(d.barrier, 0, sizeof(unsigned long long)));
+    }
     TA_TRY(cudaDeviceSynchronize());
 #undef TA_TRY
     *out = h;
@@ -414,6 +491,32 @@ int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
     const bool timed = h->timed_used < h->timed_cap;
     cudaEvent_t *ev = timed ? &h->events[4 * (size_t)h->timed_used] : nullptr;
     if (timed) cudaEventRecord(ev[0], s);
+
+    if (h->fused_ok) {
+        ta::FusedArgs fa{};
+        fa.sweep.items = d.items; fa.sweep.n_items = h->n_items; fa.sweep.n_batches = h->n_batches;
+        fa.sweep.g = g; fa.sweep.hz = Hz; fa.sweep.n_total = h->n_total; fa.sweep.seed = probe_seed; fa.sweep.step = (uint32_t)step;
+        fa.sweep.p_s1 = d.p_s1; fa.sweep.p_s2 = d.p_s2; fa.sweep.p_sa = d.p_sa;
+        fa.sweep.p_amax = d.p_amax; fa.sweep.p_amin = d.p_amin; fa.sweep.p_bad = d.p_bad;
+        fa.apply = ta::ApplyArgs{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status};
+        fa.item_lo = d.item_lo; fa.seg_len = d.seg_len; fa.verdict = d.verdict;
+        fa.state = d.state; fa.status = d.status;
+        fa.dp.hp = hyper_of(h->hp); fa.dp.eta0 = h->hp.eta0; fa.dp.has_hz = Hz ? 1u : 0u;
+        fa.dp.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; fa.dp.topk = 0u;
+        fa.L = h->L; fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base;
+        static const bool prefetch = getenv("TRIACCEL_FUSED_PREFETCH") ? atoi(getenv("TRIACCEL_FUSED_PREFETCH")) != 0 : true;
+        fa.prefetch_w = prefetch ? 1u : 0u;
+        const int grid = (int)std::min<long long>(h->fused_grid[bf16][p_index(P)], h->n_batches);
+        void *args[] = {&fa};
+        TA_CUDA(h, cudaLaunchCooperativeKernel(fused_kernel(P, bf16), dim3(grid), dim3(ta::kThreads), args, (size_t)h->L * 8, s));
+        h->barrier_base += 2ull * (unsigned long long)grid;
+        ++h->launches;
+        if (timed) { cudaEventRecord(ev[1], s); cudaEventRecord(ev[2], s); cudaEventRecord(ev[3], s); ++h->timed_used; }
+        h->stepped = true;
+        h->last_step = step;
+        h->last_stream = s;
+        return TA_OK;
+    }
 
     ta::SweepArgs sa{};
     sa.items = d.items; sa.n_items = h->n_items; sa.n_batches = h->n_batches;
@@ -556,7 +659,7 @@ int ta_stats(ta_handle *h, ta_layer_stats *out_host, ta_step_status *status)
         status->skipped = s.skipped;
         status->near_threshold_count = s.near_count;
     }
-    return TA_OK;
+    return check_device_error(h);
 }
 
 int ta_precision_codes(ta_handle *h, uint8_t *out_host)
