@@ -575,6 +575,7 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     }
     double s1 = 0.0, s2 = 0.0, sa = 0.0, bad = 0.0;
     uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+#pragma unroll 4
     for (uint32_t i = lo + tid; i < hi; i += kThreads) {
         s1 += A.p_s1[i];
         s2 += A.p_s2[i];
@@ -793,7 +794,7 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
     extern __shared__ unsigned char dyn_smem[];
     float *sh_eta = reinterpret_cast<float *>(dyn_smem);                 // [L]
     uint32_t *sh_code = reinterpret_cast<uint32_t *>(dyn_smem) + A.L;    // [L]
-    __shared__ double red[kWarps];
+    __shared__ double red[kWarps], red2[kWarps];
     __shared__ uint32_t red_u[2][kWarps];
     const uint32_t tid = threadIdx.x;
     const unsigned long long G = gridDim.x;
@@ -804,7 +805,58 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
         sweep_batch<P, BF16, false>(A.sweep, batch, nullptr);
     if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) return;
 
-    // DRAM is idle until the update starts: pull this block's weights into L2 meanwhile
+    // phase 2: blocks share the layers.  The owner of a layer combines the layer's item partials in a fixed
+    // order, takes the layer's decisions, keeps the new state in registers and publishes step size, code and
+    // its non-finite flag for everybody.  At most kOwned layers per block.
+    constexpr int kOwned = 4;
+    LayerState mine[kOwned];
+    uint32_t n_owned = 0;
+    for (uint32_t l = blockIdx.x; l < A.L; l += gridDim.x) {
+        const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
+        // thread 0 fetches what it needs for the decision while the partials are on their way
+        LayerState old;
+        double n = 1.0;
+        if (tid == 0) { old = A.state[l]; n = (double)A.seg_len[l]; }
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
+#pragma unroll 4
+        for (uint32_t i = lo + tid; i < hi; i += kThreads) {
+            s1 += __ldcg(A.sweep.p_s1 + i);
+            s2 += __ldcg(A.sweep.p_s2 + i);
+            bad |= __ldcg(A.sweep.p_bad + i);
+            if (P > 0) {
+                amax = max(amax, __ldcg(A.sweep.p_amax + i));
+                amin = min(amin, __ldcg(A.sweep.p_amin + i));
+            }
+        }
+        s1 = warp_sum(s1);
+        s2 = warp_sum(s2);
+        amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+        amin = __reduce_min_sync(0xFFFFFFFFu, amin);
+        __syncthreads();
+        if ((tid & 31) == 0) { red[tid >> 5] = s1; red2[tid >> 5] = s2; red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
+        bad = (uint32_t)__syncthreads_or((int)bad);
+        if (tid == 0) {
+            s1 = 0.0; s2 = 0.0;
+            for (int w = 0; w < kWarps; ++w) { s1 += red[w]; s2 += red2[w]; }
+            for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
+            const double mu = s1 / n;
+            double var = s2 / n - mu * mu;
+            if (!(var > 0.0)) var = 0.0;
+            LayerScratch sc;
+            sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = bad; sc.amax = amax; sc.amin = amin;
+            uint32_t near;
+            const LayerState st = decide_layer(A.dp, old, sc, near);
+            if (n_owned < (uint32_t)kOwned) mine[n_owned] = st;
+            LayerVerdict v;
+            v.eta = st.eta;
+            v.code_bad = st.code | (bad ? 0x80000000u : 0u);
+            A.verdict[l] = v;
+            if (near) atomicAdd(&A.status->near_stage, 1u);
+        }
+        ++n_owned;
+    }
+    // DRAM is idle until the update starts: pull this block's weights into L2 while waiting
     if (A.prefetch_w) {
         for (uint32_t batch = blockIdx.x; batch < A.sweep.n_batches; batch += gridDim.x) {
             const uint32_t it = batch * kWarps + (tid >> 5);
@@ -817,51 +869,6 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
         }
     }
 
-    // phase 2: blocks share the layers.  The owner of a layer combines the layer's item partials in a fixed
-    // order, takes the layer's decisions, keeps the new state in registers and publishes step size, code and
-    // its non-finite flag for everybody.  At most kOwned layers per block.
-    constexpr int kOwned = 4;
-    LayerState mine[kOwned];
-    uint32_t n_owned = 0;
-    for (uint32_t l = blockIdx.x; l < A.L; l += gridDim.x) {
-        const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
-        double s1 = 0.0, s2 = 0.0;
-        uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
-        for (uint32_t i = lo + tid; i < hi; i += kThreads) {
-            s1 += __ldcg(A.sweep.p_s1 + i);
-            s2 += __ldcg(A.sweep.p_s2 + i);
-            bad |= __ldcg(A.sweep.p_bad + i);
-            if (P > 0) {
-                amax = max(amax, __ldcg(A.sweep.p_amax + i));
-                amin = min(amin, __ldcg(A.sweep.p_amin + i));
-            }
-        }
-        s1 = block_sum(s1, red);
-        s2 = block_sum(s2, red);
-        amax = __reduce_max_sync(0xFFFFFFFFu, amax);
-        amin = __reduce_min_sync(0xFFFFFFFFu, amin);
-        bad = (uint32_t)__syncthreads_or((int)bad);
-        if ((tid & 31) == 0) { red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
-        __syncthreads();
-        if (tid == 0) {
-            for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
-            const double n = (double)A.seg_len[l];
-            const double mu = s1 / n;
-            double var = s2 / n - mu * mu;
-            if (!(var > 0.0)) var = 0.0;
-            LayerScratch sc;
-            sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = bad; sc.amax = amax; sc.amin = amin;
-            uint32_t near;
-            const LayerState st = decide_layer(A.dp, A.state[l], sc, near);
-            if (n_owned < (uint32_t)kOwned) mine[n_owned] = st;
-            LayerVerdict v;
-            v.eta = st.eta;
-            v.code_bad = st.code | (bad ? 0x80000000u : 0u);
-            A.verdict[l] = v;
-            if (near) atomicAdd(&A.status->near_stage, 1u);
-        }
-        ++n_owned;
-    }
     if (!grid_barrier(A.barrier, A.barrier_base + 2ull * G, A.status)) return;
 
     // every block reads all verdicts: is the step committed, and with which step sizes and codes

@@ -174,7 +174,7 @@ const void *fused_kernel(int P, bool bf16)
 uint64_t fused_max_params()
 {
     if (const char *env = getenv("TRIACCEL_FUSED_MAX_PARAMS")) return (uint64_t)atoll(env);
-    return 16ull << 20;
+    return 16ull << 20;      // models up to ~16 M parameters (ResNet-18 scale) take the one-launch path
 }
 
 // A bounded wait inside a kernel ran out (a block of a cooperative launch never arrived): the step that
