@@ -764,7 +764,7 @@ struct FusedArgs {
     uint32_t prefetch_w;
 };
 
-constexpr uint32_t kBarrierSpinLimit = 1u << 22;     // with a 64 ns back-off: gives up after roughly a second
+constexpr uint32_t kBarrierSpinLimit = 1u << 20;     // with a 64 ns back-off: gives up after a few hundred milliseconds
 
 // Grid-wide barrier on a monotonic arrival counter.  Returns false when the wait ran out.
 __device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsigned long long target, Status *status)

@@ -57,6 +57,7 @@ struct ta_handle {
     std::vector<cudaEvent_t> events;      // 4 per timed step: before sweep, after sweep, after decisions, after update
     uint32_t timed_cap = 0, timed_used = 0;
     // top-k: the per-layer resolve kernel runs beside the update kernel on a stream of its own
+    bool expire_next_wait = false;        // test aid: the next one-launch step waits for arrivals that never come
     bool fused_ok = false;                // small dense models: sweep + decisions + update in one cooperative launch
     int fused_grid[2][5] = {};            // resident grid of each k_fused variant: [bf16][index of P in 0,1,2,4,8]
     unsigned long long barrier_base = 0;  // barrier arrivals of all fused launches so far
@@ -441,6 +442,14 @@ int ta_launch_count(ta_handle *h, uint64_t *count)
     return TA_OK;
 }
 
+int ta_test_expire_next_wait(ta_handle *h)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!h->fused_ok) return fail(h, TA_ERR_STATE, "ta_test_expire_next_wait: this handle does not use the one-launch path");
+    h->expire_next_wait = true;
+    return TA_OK;
+}
+
 int ta_timing_begin(ta_handle *h, uint32_t max_steps)
 {
     if (!h) return TA_ERR_ARG;
@@ -504,6 +513,7 @@ int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
         fa.dp.hp = hyper_of(h->hp); fa.dp.eta0 = h->hp.eta0; fa.dp.has_hz = Hz ? 1u : 0u;
         fa.dp.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; fa.dp.topk = 0u;
         fa.L = h->L; fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base;
+        if (h->expire_next_wait) { fa.barrier_base += 1ull << 40; h->expire_next_wait = false; }
         static const bool prefetch = getenv("TRIACCEL_FUSED_PREFETCH") ? atoi(getenv("TRIACCEL_FUSED_PREFETCH")) != 0 : true;
         fa.prefetch_w = prefetch ? 1u : 0u;
         const int grid = (int)std::min<long long>(h->fused_grid[bf16][p_index(P)], h->n_batches);
@@ -669,7 +679,7 @@ int ta_precision_codes(ta_handle *h, uint8_t *out_host)
     std::vector<ta::LayerState> st(h->L);
     TA_CUDA(h, cudaMemcpy(st.data(), h->d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost));
     for (uint32_t l = 0; l < h->L; ++l) out_host[l] = (uint8_t)st[l].code;
-    return TA_OK;
+    return check_device_error(h);
 }
 
 int ta_masks(ta_handle *h, const uint32_t **dev_bits, uint64_t *num_words)

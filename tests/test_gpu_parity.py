@@ -313,3 +313,30 @@ def test_learning_rate_schedule_and_control_interval():
         sigma = 1e-5 if t < 4 else 1.0
         g = torch.from_numpy((rng.standard_normal(n_total) * sigma).astype(np.float32)).cuda()
         run.step(t, g, oracle_hz(D, 1, 3, t) if t != 2 else None, 3)
+
+
+def test_bounded_wait_runs_out_without_hanging():
+    # the one-launch path waits at grid barriers; a wait that cannot be satisfied must end by itself,
+    # leave everything untouched, be reported once, and leave the handle usable
+    wl = W.get("mlp_tiny")
+    g1, g2 = W.make_grads(wl, 1, "cuda"), W.make_grads(wl, 2, "cuda")
+    hs, ws, cs = [], [], []
+    for _ in range(2):
+        hs.append(ta.ta_create(wl.table, wl.n_total, **wl.hparams()))
+        ws.append(W.make_weights(wl, "cuda"))
+        cs.append(torch.zeros(wl.n_total, dtype=torch.int16, device="cuda"))
+        ta.ta_step(hs[-1], ws[-1], g1, None, cs[-1], 0, 1)
+    ta.ta_stats(hs[0])
+    before = (ws[0].clone(), cs[0].clone(), [(s.ema_var, s.code) for s in ta.ta_stats(hs[0])[0]])
+    ta.ta_test_expire_next_wait(hs[0])
+    ta.ta_step(hs[0], ws[0], g2, None, cs[0], 0, 2)              # every block gives up at the first barrier
+    with pytest.raises(ta.TriAccelError) as e:
+        ta.ta_stats(hs[0])
+    assert e.value.code == ta.TA_ERR_CUDA and "wait ran out" in str(e.value)
+    assert torch.equal(ws[0].view(torch.int32), before[0].view(torch.int32)) and torch.equal(cs[0], before[1])
+    assert [(s.ema_var, s.code) for s in ta.ta_stats(hs[0])[0]] == before[2]      # reported once; state untouched
+    # both handles now take the same next step and must agree bit for bit
+    ta.ta_step(hs[0], ws[0], g2, None, cs[0], 0, 3)
+    ta.ta_step(hs[1], ws[1], g2, None, cs[1], 0, 3)
+    assert torch.equal(ws[0].view(torch.int32), ws[1].view(torch.int32)) and torch.equal(cs[0], cs[1])
+    assert ta.ta_stats(hs[0])[1].skipped == 0
