@@ -61,6 +61,10 @@ struct ta_handle {
     bool fused_ok = false;                // small dense models: sweep + decisions + update in one cooperative launch
     int fused_grid[2][5] = {};            // resident grid of each k_fused variant: [bf16][index of P in 0,1,2,4,8]
     unsigned long long barrier_base = 0;  // barrier arrivals of all fused launches so far
+    std::vector<ta::Item> items_host;     // the plan, kept for the pipelined host path
+    cudaStream_t copy_back = nullptr;     // ta_step_host: device-to-host copies run beside the host-to-device ones
+    std::vector<cudaEvent_t> chunk_done;
+    cudaEvent_t decided = nullptr;
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     DeviceBuffers d;
@@ -154,6 +158,18 @@ template <bool BF16> bool dispatch_sweep(ta_handle *h, int P, const ta::SweepArg
     case 8: topk ? launch_sweep<8, BF16, true>(h, a, s) : launch_sweep<8, BF16, false>(h, a, s); return true;
     default: return false;
     }
+}
+
+// Update + cast over the items [item_begin, item_begin + item_count) (item_begin a multiple of the batch size).
+void launch_apply(ta_handle *h, float *w, const void *g, uint16_t *c, uint32_t item_begin, uint32_t item_count, cudaStream_t s)
+{
+    if (item_count == 0) return;
+    const uint32_t batches = (item_count + ta::kWarps - 1) / ta::kWarps;
+    ta::ApplyArgs aa{h->d.items + item_begin, item_count, batches, w, g, c, h->d.state, h->d.status};
+    const int grid = (int)std::min<long long>(batches, (long long)h->sm_count * 8);
+    if (h->hp.grad_dtype == TA_GRAD_BF16) ta::k_apply<true><<<grid, ta::kThreads, 0, s>>>(aa);
+    else ta::k_apply<false><<<grid, ta::kThreads, 0, s>>>(aa);
+    ++h->launches;
 }
 
 int p_index(int P) { return P == 0 ? 0 : P == 1 ? 1 : P == 2 ? 2 : P == 4 ? 3 : 4; }
@@ -334,6 +350,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         if (items.size() > 0x7FFFFFFFull) { snprintf(h->err, 256, "ta_create: too many work items"); return bail(TA_ERR_ARG); }
     }
     item_lo[L] = (uint32_t)items.size();
+    h->items_host = items;
     h->n_items = (uint32_t)items.size();
     h->n_batches = (h->n_items + ta::kWarps - 1) / ta::kWarps;
     if (h->fused_ok && std::min<long long>(fused_blocks, h->n_batches) * 4 < (long long)L) h->fused_ok = false;
@@ -419,6 +436,9 @@ int ta_destroy(ta_handle *h)
     if (h->last_stream || h->stepped) cudaStreamSynchronize(h->last_stream);
     for (cudaEvent_t e : h->events) cudaEventDestroy(e);
     if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
+    if (h->copy_back) { cudaStreamSynchronize(h->copy_back); cudaStreamDestroy(h->copy_back); }
+    for (cudaEvent_t e : h->chunk_done) cudaEventDestroy(e);
+    if (h->decided) cudaEventDestroy(h->decided);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     free_all(h->d);
@@ -482,8 +502,10 @@ int ta_timing_end(ta_handle *h, double *ms_sweep, double *ms_decide, double *ms_
     return TA_OK;
 }
 
-int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c, uint64_t probe_seed, uint64_t step,
-            void *stream)
+// The whole step; with defer_apply the update kernel is left to the caller (launch_apply), who may run it
+// piecewise while the weights are still arriving from the host.
+static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c, uint64_t probe_seed,
+                     uint64_t step, void *stream, bool defer_apply)
 {
     if (!h) return TA_ERR_ARG;
     if (!w || !g || !c) return fail(h, TA_ERR_ARG, "ta_step: w, g and c must not be NULL");
@@ -566,10 +588,7 @@ int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
     }
 
     if (timed) cudaEventRecord(ev[2], s);
-    ta::ApplyArgs aa{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status};
-    if (bf16) ta::k_apply<true><<<grid_for(h), ta::kThreads, 0, s>>>(aa);
-    else ta::k_apply<false><<<grid_for(h), ta::kThreads, 0, s>>>(aa);
-    ++h->launches;
+    if (!defer_apply) launch_apply(h, w, g, c, 0, h->n_items, s);
     if (topk) TA_CUDA(h, cudaStreamWaitEvent(s, h->ev_join, 0));
     if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
 
@@ -578,6 +597,12 @@ int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c,
     h->last_step = step;
     h->last_stream = s;
     return TA_OK;
+}
+
+int ta_step(ta_handle *h, float *w, const void *g, const float *Hz, uint16_t *c, uint64_t probe_seed, uint64_t step,
+            void *stream)
+{
+    return step_impl(h, w, g, Hz, c, probe_seed, step, stream, false);
 }
 
 int ta_step_host(ta_handle *h, float *w_host, const void *g_host, const float *Hz_host, uint16_t *c_host,
@@ -594,6 +619,63 @@ int ta_step_host(ta_handle *h, float *w_host, const void *g_host, const float *H
         TA_CUDA(h, cudaMalloc(&d.st_g, std::max<size_t>(g_bytes, 16)));
         TA_CUDA(h, dev_alloc(&d.st_c, n));
         TA_CUDA(h, dev_alloc(&d.st_hz, n * h->hp.num_probes));
+    }
+    if (!h->fused_ok && !h->topk && h->n_items >= 64 * ta::kWarps) {
+        // Large dense model: the statistics need only g and Hz, so they are copied first and the sweep and the
+        // decisions run while the weights are still on their way.  The weights then arrive in chunks; each
+        // chunk is updated as soon as it is there and travels back on a second stream while the next one comes in.
+        constexpr uint32_t kChunks = 16;
+        if (!h->copy_back) {
+            TA_CUDA(h, cudaStreamCreateWithFlags(&h->copy_back, cudaStreamNonBlocking));
+            TA_CUDA(h, cudaEventCreateWithFlags(&h->decided, cudaEventDisableTiming));
+            for (uint32_t k = 0; k < kChunks; ++k) {
+                cudaEvent_t e;
+                TA_CUDA(h, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+                h->chunk_done.push_back(e);
+            }
+        }
+        TA_CUDA(h, cudaMemcpyAsync(d.st_g, g_host, g_bytes, cudaMemcpyHostToDevice, s));
+        if (Hz_host) TA_CUDA(h, cudaMemcpyAsync(d.st_hz, Hz_host, n * 4 * h->hp.num_probes, cudaMemcpyHostToDevice, s));
+        const int rc = step_impl(h, d.st_w, d.st_g, Hz_host ? d.st_hz : nullptr, d.st_c, probe_seed, step, stream, true);
+        if (rc != TA_OK) return rc;
+        std::vector<ta::LayerState> st(h->L);
+        ta::Status status;
+        TA_CUDA(h, cudaMemcpyAsync(st.data(), d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost, s));
+        TA_CUDA(h, cudaMemcpyAsync(&status, d.status, sizeof(status), cudaMemcpyDeviceToHost, s));
+        TA_CUDA(h, cudaEventRecord(h->decided, s));
+        // chunk boundaries on whole batches of items
+        uint32_t bounds[kChunks + 1];
+        for (uint32_t k = 0; k <= kChunks; ++k)
+            bounds[k] = k == kChunks ? h->n_items : (uint32_t)((uint64_t)h->n_items * k / kChunks) / ta::kWarps * ta::kWarps;
+        auto elem_begin = [&](uint32_t k) { return h->items_host[bounds[k]].begin; };
+        auto elem_end = [&](uint32_t k) { return k + 1 == kChunks ? h->items_host.back().begin + h->items_host.back().len : h->items_host[bounds[k + 1]].begin; };
+        for (uint32_t k = 0; k < kChunks; ++k) {
+            const uint64_t b = elem_begin(k), e = elem_end(k);
+            TA_CUDA(h, cudaMemcpyAsync(d.st_w + b, w_host + b, (e - b) * 4, cudaMemcpyHostToDevice, s));
+            launch_apply(h, d.st_w, d.st_g, d.st_c, bounds[k], bounds[k + 1] - bounds[k], s);
+            TA_CUDA(h, cudaEventRecord(h->chunk_done[k], s));
+        }
+        TA_CUDA(h, cudaGetLastError());
+        TA_CUDA(h, cudaEventSynchronize(h->decided));          // codes and the skip flag are on the host now
+        if (!status.skipped) {
+            uint32_t l = 0;
+            for (uint32_t k = 0; k < kChunks; ++k) {
+                const uint64_t b = elem_begin(k), e = elem_end(k);
+                TA_CUDA(h, cudaStreamWaitEvent(h->copy_back, h->chunk_done[k], 0));
+                TA_CUDA(h, cudaMemcpyAsync(w_host + b, d.st_w + b, (e - b) * 4, cudaMemcpyDeviceToHost, h->copy_back));
+                // 16-bit copies: the parts of FP16 / BF16 layers that lie in this chunk
+                while (l < h->L && h->table[l].offset + h->table[l].length <= b) ++l;
+                for (uint32_t j = l; j < h->L && h->table[j].offset < e; ++j) {
+                    if (st[j].code >= TA_CODE_FP32) continue;
+                    const uint64_t cb = std::max<uint64_t>(b, h->table[j].offset);
+                    const uint64_t ce = std::min<uint64_t>(e, h->table[j].offset + h->table[j].length);
+                    if (ce > cb) TA_CUDA(h, cudaMemcpyAsync(c_host + cb, d.st_c + cb, (ce - cb) * 2, cudaMemcpyDeviceToHost, h->copy_back));
+                }
+            }
+        }
+        TA_CUDA(h, cudaStreamSynchronize(s));
+        TA_CUDA(h, cudaStreamSynchronize(h->copy_back));
+        return TA_OK;
     }
     TA_CUDA(h, cudaMemcpyAsync(d.st_w, w_host, n * 4, cudaMemcpyHostToDevice, s));
     TA_CUDA(h, cudaMemcpyAsync(d.st_g, g_host, g_bytes, cudaMemcpyHostToDevice, s));

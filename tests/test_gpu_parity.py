@@ -279,6 +279,34 @@ def test_step_host_matches_device_step():
         assert torch.equal(c.cpu(), ch)
 
 
+def test_step_host_pipelined_matches_device_step(monkeypatch):
+    # large dense models take the pipelined host path (statistics first, weights in chunks with overlapped
+    # copy-back); force it on a mid-size model by switching the one-launch path off
+    monkeypatch.setenv("TRIACCEL_FUSED_MAX_PARAMS", "0")
+    wl = W.get("resnet18_cifar", align=1)                  # odd offsets: chunk edges fall inside vectors
+    D = W.make_curvature(wl, "cuda")
+    z = torch.empty(wl.n_total, device="cuda")
+    a = ta.ta_create(wl.table, wl.n_total, **wl.hparams())
+    b = ta.ta_create(wl.table, wl.n_total, **wl.hparams())
+    w = W.make_weights(wl, "cuda")
+    c = torch.full((wl.n_total,), 0x1111, dtype=torch.int16, device="cuda")
+    wh = w.cpu().pin_memory()
+    ch = c.cpu().pin_memory()
+    for t in range(1, 5):
+        g = W.make_grads(wl, t, "cuda")
+        if t == 3:
+            g[wl.table[10][0] + 3] = float("nan")           # a skipped step copies nothing back
+        ta.ta_probe(a, 0, t, 0, z)
+        hz = D * z if t != 2 else None
+        ta.ta_step(a, w, g, hz, c, 0, t)
+        ta.ta_step_host(b, wh, g.cpu().pin_memory(), hz.cpu().pin_memory() if hz is not None else None, ch, 0, t)
+        assert torch.equal(w.cpu().view(torch.int32), wh.view(torch.int32)), t
+        assert torch.equal(c.cpu(), ch), t
+        sa, sb = ta.ta_stats(a), ta.ta_stats(b)
+        assert sa[1].skipped == sb[1].skipped == (1 if t == 3 else 0)
+        assert [(s.ema_var, s.code) for s in sa[0]] == [(s.ema_var, s.code) for s in sb[0]]
+
+
 def test_argument_errors_enqueue_nothing():
     n = 4096
     h = ta.ta_create([(0, n)], n)
