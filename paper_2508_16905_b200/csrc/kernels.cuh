@@ -15,6 +15,29 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Tuning constants (rows of 128 elements a lane keeps in flight).
+#ifndef TA_SWEEP_ROWS_P1
+#define TA_SWEEP_ROWS_P1 8
+#endif
+#ifndef TA_SWEEP_ROWS_P1_BF16
+#define TA_SWEEP_ROWS_P1_BF16 16
+#endif
+#ifndef TA_SWEEP_ROWS_P2
+#define TA_SWEEP_ROWS_P2 4
+#endif
+#ifndef TA_SWEEP_ROWS_P4
+#define TA_SWEEP_ROWS_P4 2
+#endif
+#ifndef TA_APPLY_ROWS
+#define TA_APPLY_ROWS 4
+#endif
+#ifndef TA_APPLY_ROWS_BF16
+#define TA_APPLY_ROWS_BF16 8
+#endif
+#ifndef TA_APPLY_STREAM_W_STORE
+#define TA_APPLY_STREAM_W_STORE 0
+#endif
+
 namespace ta {
 
 constexpr int kWarps = 8;
@@ -243,7 +266,8 @@ template <int P, bool BF16, bool TOPK>
 __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, uint32_t *sh_hist)
 {
     constexpr int PP = P > 0 ? P : 1;
-    constexpr int U = (P <= 1) ? 8 : (P == 2 ? 4 : 2);     // rows in flight per lane
+    constexpr int U = (P <= 1) ? (BF16 ? TA_SWEEP_ROWS_P1_BF16 : TA_SWEEP_ROWS_P1)
+                               : (P == 2 ? TA_SWEEP_ROWS_P2 : TA_SWEEP_ROWS_P4);     // rows in flight per lane
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     {
         const uint32_t it = batch * kWarps + warp;
@@ -651,7 +675,7 @@ __device__ __forceinline__ uint16_t cast16(float x, uint32_t code)
 template <bool BF16, typename Decision>
 __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, const Decision &decision)
 {
-    constexpr int U = 4;
+    constexpr int U = BF16 ? TA_APPLY_ROWS_BF16 : TA_APPLY_ROWS;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     {
         const uint32_t it = batch * kWarps + warp;
@@ -680,7 +704,8 @@ __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, 
             wv.y = fmaf(neg_eta, gv.y, wv.y);
             wv.z = fmaf(neg_eta, gv.z, wv.z);
             wv.w = fmaf(neg_eta, gv.w, wv.w);
-            *reinterpret_cast<float4 *>(A.w + i0) = wv;
+            if (TA_APPLY_STREAM_W_STORE) __stcs(reinterpret_cast<float4 *>(A.w + i0), wv);
+            else *reinterpret_cast<float4 *>(A.w + i0) = wv;
             if (code == 0u) {
                 const __half2 a = __floats2half2_rn(wv.x, wv.y), b = __floats2half2_rn(wv.z, wv.w);
                 uint2 o;
