@@ -188,6 +188,34 @@ int ta_precision_codes(ta_handle *h, uint8_t *out_host);
  */
 int ta_masks(ta_handle *h, const uint32_t **dev_bits, uint64_t *num_words);
 
+/*
+ * ta_power_iterate -- one step of the per-layer power iteration of Sec. 3.2,
+ *     u <- H_l u / ||H_l u||,   lambda ~ (u^T H_l u) / (u^T u),
+ * for all layers at once, on the same flat layout.  The caller supplies the products Hu (per layer, the
+ * block H_l applied to u_l; e.g. from autograd).  To find the top-k eigenvalues one after the other (the
+ * paper uses k = 5), eigenvectors already found are deflated:  Hu' = Hu - sum_j lambda_j (v_j . u) v_j.
+ *   u, Hu      device float[n_total]
+ *   V          device float[m][n_total], unit eigenvectors found so far (NULL when m = 0)
+ *   lambda_V   device float[m][L], their eigenvalues per layer (NULL when m = 0)
+ *   m          number of deflated vectors, <= TA_MAX_EIGS
+ *   u_next     device float[n_total] (output; may be u itself): Hu' / ||Hu'|| per layer, 0 where ||Hu'|| = 0
+ *   lambda_out device float[L] (output): Rayleigh quotient u . Hu' / u . u per layer (0 where u = 0)
+ *   norm_out   device float[L] (output) or NULL: ||Hu'|| per layer
+ * Sums are double, combined in a fixed order (bit-reproducible).  Asynchronous on `stream`.
+ * Errors: TA_ERR_ARG, TA_ERR_ALIGN, TA_ERR_NOMEM (workspace, allocated at the first call), TA_ERR_CUDA.
+ */
+#define TA_MAX_EIGS 8
+int ta_power_iterate(ta_handle *h, const float *u, const float *Hu, const float *V, const float *lambda_V, uint32_t m,
+                     float *u_next, float *lambda_out, float *norm_out, void *stream);
+
+/*
+ * ta_set_curvature -- sets lambda_l of every layer from host values (e.g. the largest of the top-k
+ * eigenvalues found by ta_power_iterate: max_{i<=k} lambda_i(H_l), Sec. 3.2).  The following ta_step calls
+ * with Hz = NULL use them for the step size and the precision promotion.  Waits for the stream.
+ * Errors: TA_ERR_ARG (NULL, negative or non-finite value), TA_ERR_CUDA.
+ */
+int ta_set_curvature(ta_handle *h, const float *lambda_max_host);
+
 /* Number of kernels the library launched on behalf of this handle so far (for benchmarks). */
 int ta_launch_count(ta_handle *h, uint64_t *count);
 

@@ -65,6 +65,8 @@ def lib():
         L.orc_cast_array.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p]
         L.orc_hutchinson_abs.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint64,
                                          C.c_uint64, C.c_uint64, C.c_void_p]
+        L.orc_power_iterate.argtypes = [C.POINTER(Segment), C.c_uint32, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_batch_next.restype = C.c_int64
         L.orc_batch_next.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_double, C.c_double,
                                      C.c_double, C.c_double, C.c_int64, C.c_int64]
@@ -117,6 +119,25 @@ def hutchinson_abs(hz, n_total, P, seed, t, offset, length):
     a = np.empty(length, dtype=np.float32)
     lib().orc_hutchinson_abs(_ptr(hz), n_total, P, seed, t, offset, length, _ptr(a))
     return a
+
+
+def power_iterate(table, n_total, u, hu, v=None, lam_v=None):
+    """One power-iteration step per layer. v: [m, n_total] or None; lam_v: [m, L] or None.
+    Returns (u_next [n_total], lambda [L], norm [L]); elements outside the layers of u_next are 0."""
+    L = len(table)
+    segs = (Segment * L)(*[Segment(int(o), int(n)) for o, n in table])
+    u = np.ascontiguousarray(u, dtype=np.float32)
+    hu = np.ascontiguousarray(hu, dtype=np.float32)
+    m = 0 if v is None else int(np.asarray(v).shape[0])
+    if m:
+        v = np.ascontiguousarray(v, dtype=np.float32).reshape(m, n_total)
+        lam_v = np.ascontiguousarray(lam_v, dtype=np.float32).reshape(m, L)
+    out = np.zeros(n_total, dtype=np.float32)
+    lam = np.zeros(L, dtype=np.float32)
+    nrm = np.zeros(L, dtype=np.float32)
+    lib().orc_power_iterate(segs, L, n_total, _ptr(u), _ptr(hu), _ptr(v) if m else None, _ptr(lam_v) if m else None, m,
+                            _ptr(out), _ptr(lam), _ptr(nrm))
+    return out, lam, nrm
 
 
 def batch_next(B, delta_up, delta_down, rho_low, rho_high, mem_usage, mem_max, B_min, B_max):

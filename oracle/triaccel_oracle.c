@@ -23,6 +23,7 @@
  *   control interval       Sec. 3.4, decisions every T_ctrl steps
  *   master update + cast   Sec. 2 (FP32 master copy, low-precision working copy),
  *                          Sec. 3.2 (per-layer step size), Sec. 4.1 (SGD)
+ *   orc_power_iterate      Sec. 3.2, u <- H u / ||H u||, lambda ~ u^T H u / u^T u (with deflation for top-k)
  *   orc_batch_next         Sec. 3.3, the three-branch rule for B(t+1)
  *   orc_philox4x32_10      Salmon, Moraes, Dror, Shaw: "Parallel random numbers:
  *                          as easy as 1, 2, 3" (SC'11), Philox-4x32, 10 rounds.
@@ -32,7 +33,7 @@
  * Pins (tests/, CPU only): Philox known-answer vectors; exact rational brute
  * force for the moments; EMA closed form; Hz = D*z  =>  estimate == D;
  * all 2^n sign vectors on a dense symmetric H; full-sort brute force for the
- * mask; exhaustive rounding-class enumeration of both casts against numpy /
+ * mask; power iteration against a dense symmetric eigensolver; exhaustive rounding-class enumeration of both casts against numpy /
  * torch conversions; boundary and monotonicity cases of the code rule.
  * Unpinned: the end-to-end trajectory over many steps (the paper prints no
  * worked example); it is pinned only through its parts.
@@ -430,6 +431,45 @@ int orc_step(orc_state *st, float *w, const void *g_any, const float *hz, uint16
     }
     free(gl); free(a); free(cand);
     return 0;
+}
+
+/* ---------------------------------------------------------------- power iteration (Sec. 3.2) */
+
+/*
+ * One step of u <- H_l u / ||H_l u||, lambda ~ u^T H_l u / u^T u for every layer, with the products hu = H_l u
+ * given.  m earlier eigenvectors v[j] (flat, [m][n_total]) with per-layer eigenvalues lam_v[j*L + l] are
+ * deflated: t = hu - sum_j a_j v_j, a_j = float(lam_j * (v_j . u)), subtracted one after the other with one
+ * float rounding each (fused multiply-add), in the order j = 0, 1, ...
+ */
+void orc_power_iterate(const orc_segment *table, uint32_t L, uint64_t n_total, const float *u, const float *hu,
+                       const float *v, const float *lam_v, uint32_t m, float *u_next, float *lambda_out, float *norm_out)
+{
+    for (uint32_t l = 0; l < L; ++l) {
+        const uint64_t off = table[l].offset, n = table[l].length;
+        float a[8];
+        for (uint32_t j = 0; j < m; ++j) {
+            double dot = 0.0;
+            for (uint64_t i = 0; i < n; ++i) dot += (double)v[(uint64_t)j * n_total + off + i] * (double)u[off + i];
+            a[j] = (float)((double)lam_v[(uint64_t)j * L + l] * dot);
+        }
+        double uu = 0.0, ut = 0.0, tt = 0.0;
+        for (uint64_t i = 0; i < n; ++i) {
+            float t = hu[off + i];
+            for (uint32_t j = 0; j < m; ++j) t = fmaf(-a[j], v[(uint64_t)j * n_total + off + i], t);
+            uu += (double)u[off + i] * (double)u[off + i];
+            ut += (double)u[off + i] * (double)t;
+            tt += (double)t * (double)t;
+        }
+        const float nrm = (float)sqrt(tt);
+        lambda_out[l] = uu > 0.0 ? (float)(ut / uu) : 0.0f;
+        if (norm_out) norm_out[l] = nrm;
+        for (uint64_t i = 0; i < n; ++i) {
+            float t = hu[off + i];
+            for (uint32_t j = 0; j < m; ++j) t = fmaf(-a[j], v[(uint64_t)j * n_total + off + i], t);
+            volatile float q = nrm > 0.0f ? t / nrm : 0.0f;
+            u_next[off + i] = q;
+        }
+    }
 }
 
 /* ---------------------------------------------------------------- batch rule */

@@ -20,7 +20,8 @@ TA_GRAD_F32, TA_GRAD_BF16 = 0, 1
 EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "ta_probe", "ta_stats",
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
            "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
-           "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait"]
+           "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait",
+           "ta_power_iterate", "ta_set_curvature"]
 
 
 class ta_segment(C.Structure):
@@ -93,6 +94,8 @@ def lib():
     L.ta_timing_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(u32)]
     L.ta_grad_moments_static.argtypes = [C.POINTER(ta_segment), u32, vp, u32, vp, vp, vp]
     L.ta_test_expire_next_wait.argtypes = [vp]
+    L.ta_power_iterate.argtypes = [vp, vp, vp, vp, vp, u32, vp, vp, vp, vp]
+    L.ta_set_curvature.argtypes = [vp, vp]
     L.ta_static_last_error.argtypes = []
     L.ta_static_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -253,6 +256,18 @@ def ta_grad_moments_static(table, g, grad_dtype, mean_var, nonfinite=None, strea
     rc = lib().ta_grad_moments_static(segs, L, _dev_ptr(g), gd, _dev_ptr(mean_var), _dev_ptr(nonfinite), _stream(stream))
     if rc != TA_OK:
         raise TriAccelError(rc, (lib().ta_static_last_error() or b"").decode())
+
+
+def ta_power_iterate(h, u, Hu, V, lambda_V, m, u_next, lambda_out, norm_out=None, stream=None):
+    _check(lib().ta_power_iterate(h.ptr, _dev_ptr(u), _dev_ptr(Hu), _dev_ptr(V), _dev_ptr(lambda_V), int(m),
+                                  _dev_ptr(u_next), _dev_ptr(lambda_out), _dev_ptr(norm_out), _stream(stream)), h.ptr)
+
+
+def ta_set_curvature(h, lambda_max):
+    a = np.ascontiguousarray(lambda_max, dtype=np.float32)
+    if a.size != h.L:
+        raise ValueError("one value per layer")
+    _check(lib().ta_set_curvature(h.ptr, a.ctypes.data_as(C.c_void_p)), h.ptr)
 
 
 def ta_test_expire_next_wait(h):

@@ -934,6 +934,150 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
     for (uint32_t batch = blockIdx.x; batch < A.apply.n_batches; batch += gridDim.x) apply_batch<BF16>(A.apply, batch, decision);
 }
 
+// ------------------------------------------------------------------ power iteration support (Sec. 3.2)
+//
+// u <- H_l u / ||H_l u||,  lambda ~ (u^T H_l u) / (u^T u), per layer, with the products H_l u supplied by the
+// caller.  Eigenvectors found earlier (V, with eigenvalues lambda_V) are deflated:
+//   t = Hu - sum_j a_j v_j,   a_j = lambda_j (v_j . u)   per layer.
+// Three sweeps over the same items as the optimizer pass: projections v_j . u, then the dots of u and t, then
+// the normalised write.  All sums are double and combined in a fixed order.
+
+constexpr int kMaxEigs = 8;
+
+struct PowerArgs {
+    const Item *items;
+    uint32_t n_items, n_batches;
+    const float *u, *hu, *v;       // v: [m][n_total]
+    uint64_t n_total;
+    uint32_t m, L;
+    double *part;                  // [max(3, m)][n_items] per-item partial sums
+    const float *coef;             // [kMaxEigs][L] a_j per layer
+    const float *norm;             // [L]
+    float *u_next;
+};
+
+__device__ __forceinline__ float4 load_row4(const float *p, uint64_t i0, bool full, uint64_t begin, uint64_t end)
+{
+    if (full) return __ldg(reinterpret_cast<const float4 *>(p + i0));
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i0 + 0 >= begin && i0 + 0 < end) r.x = __ldg(p + i0 + 0);
+    if (i0 + 1 >= begin && i0 + 1 < end) r.y = __ldg(p + i0 + 1);
+    if (i0 + 2 >= begin && i0 + 2 < end) r.z = __ldg(p + i0 + 2);
+    if (i0 + 3 >= begin && i0 + 3 < end) r.w = __ldg(p + i0 + 3);
+    return r;
+}
+
+// MODE 0: projections v_j . u;  MODE 1: u.u, u.t, t.t;  MODE 2: u_next = t / ||t||
+template <int MODE>
+__global__ void __launch_bounds__(kThreads) k_power(const PowerArgs A)
+{
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+        const uint32_t it = batch * kWarps + warp;
+        if (it >= A.n_items) continue;
+        const Item item = A.items[it];
+        double acc[kMaxEigs];
+#pragma unroll
+        for (int j = 0; j < kMaxEigs; ++j) acc[j] = 0.0;
+        if (item.len != 0u) {
+            const uint64_t begin = item.begin, end = begin + item.len;
+            float a[kMaxEigs];
+#pragma unroll
+            for (int j = 0; j < kMaxEigs; ++j) a[j] = (MODE != 0 && j < (int)A.m) ? A.coef[(uint64_t)j * A.L + item.seg] : 0.f;
+            const float nrm = MODE == 2 ? A.norm[item.seg] : 1.f;
+            const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
+            for (uint64_t row = row_first; row <= row_last; ++row) {
+                const uint64_t i0 = row * 128ull + lane * 4u;
+                const bool full = row * 128ull >= begin && row * 128ull + 128u <= end;
+                if (MODE == 0) {
+                    const float4 uu = load_row4(A.u, i0, full, begin, end);
+#pragma unroll
+                    for (int j = 0; j < kMaxEigs; ++j) {
+                        if (j < (int)A.m) {
+                            const float4 vv = load_row4(A.v + (uint64_t)j * A.n_total, i0, full, begin, end);
+                            acc[j] += (double)vv.x * (double)uu.x + (double)vv.y * (double)uu.y +
+                                      (double)vv.z * (double)uu.z + (double)vv.w * (double)uu.w;
+                        }
+                    }
+                } else {
+                    float4 t = load_row4(A.hu, i0, full, begin, end);
+#pragma unroll
+                    for (int j = 0; j < kMaxEigs; ++j) {
+                        if (j < (int)A.m) {
+                            const float4 vv = load_row4(A.v + (uint64_t)j * A.n_total, i0, full, begin, end);
+                            t.x = fmaf(-a[j], vv.x, t.x); t.y = fmaf(-a[j], vv.y, t.y);
+                            t.z = fmaf(-a[j], vv.z, t.z); t.w = fmaf(-a[j], vv.w, t.w);
+                        }
+                    }
+                    if (MODE == 1) {
+                        const float4 uu = load_row4(A.u, i0, full, begin, end);
+                        acc[0] += (double)uu.x * (double)uu.x + (double)uu.y * (double)uu.y + (double)uu.z * (double)uu.z + (double)uu.w * (double)uu.w;
+                        acc[1] += (double)uu.x * (double)t.x + (double)uu.y * (double)t.y + (double)uu.z * (double)t.z + (double)uu.w * (double)t.w;
+                        acc[2] += (double)t.x * (double)t.x + (double)t.y * (double)t.y + (double)t.z * (double)t.z + (double)t.w * (double)t.w;
+                    } else {
+                        float4 o;
+                        o.x = nrm > 0.f ? __fdiv_rn(t.x, nrm) : 0.f; o.y = nrm > 0.f ? __fdiv_rn(t.y, nrm) : 0.f;
+                        o.z = nrm > 0.f ? __fdiv_rn(t.z, nrm) : 0.f; o.w = nrm > 0.f ? __fdiv_rn(t.w, nrm) : 0.f;
+                        if (full) {
+                            *reinterpret_cast<float4 *>(A.u_next + i0) = o;
+                        } else {
+                            if (i0 + 0 >= begin && i0 + 0 < end) A.u_next[i0 + 0] = o.x;
+                            if (i0 + 1 >= begin && i0 + 1 < end) A.u_next[i0 + 1] = o.y;
+                            if (i0 + 2 >= begin && i0 + 2 < end) A.u_next[i0 + 2] = o.z;
+                            if (i0 + 3 >= begin && i0 + 3 < end) A.u_next[i0 + 3] = o.w;
+                        }
+                    }
+                }
+            }
+        }
+        if (MODE != 2) {
+            const int n_acc = MODE == 0 ? (int)A.m : 3;
+#pragma unroll
+            for (int j = 0; j < kMaxEigs; ++j) {
+                if (j < n_acc) {
+                    const double v = warp_sum(acc[j]);
+                    if (lane == 0) A.part[(uint64_t)j * A.n_items + it] = v;
+                }
+            }
+        }
+    }
+}
+
+struct PowerLayerArgs {
+    const uint32_t *item_lo;
+    uint32_t n_items, m, L;
+    const double *part;
+    const float *lambda_v;         // [m][L] eigenvalues of the deflated vectors
+    float *coef;                   // [kMaxEigs][L]
+    float *lambda_out, *norm_out;  // [L]
+};
+
+// One block per layer.  STAGE 0: a_j = lambda_j * (v_j . u).  STAGE 1: lambda = u.t / u.u, norm = sqrt(t.t).
+template <int STAGE>
+__global__ void __launch_bounds__(kThreads) k_power_layer(const PowerLayerArgs A)
+{
+    __shared__ double red[kWarps];
+    const uint32_t l = blockIdx.x, tid = threadIdx.x;
+    const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
+    const int n_acc = STAGE == 0 ? (int)A.m : 3;
+    double tot[3] = {0.0, 0.0, 0.0};
+    for (int j = 0; j < n_acc; ++j) {
+        double sum = 0.0;
+#pragma unroll 4
+        for (uint32_t i = lo + tid; i < hi; i += kThreads) sum += A.part[(uint64_t)j * A.n_items + i];
+        sum = block_sum(sum, red);
+        if (STAGE == 0) {
+            if (tid == 0) A.coef[(uint64_t)j * A.L + l] = (float)((double)A.lambda_v[(uint64_t)j * A.L + l] * sum);
+        } else {
+            tot[j] = sum;
+        }
+    }
+    if (STAGE == 1 && tid == 0) {
+        A.lambda_out[l] = tot[0] > 0.0 ? (float)(tot[1] / tot[0]) : 0.f;
+        A.norm_out[l] = (float)sqrt(tot[2]);
+    }
+}
+
 // ------------------------------------------------------------------ probe writer
 
 __global__ void __launch_bounds__(kThreads) k_probe(float *z, uint64_t n_vec, uint64_t seed, uint32_t step, uint32_t p)

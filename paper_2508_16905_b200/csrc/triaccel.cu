@@ -31,6 +31,9 @@ struct DeviceBuffers {
     ta::SelectState *sel = nullptr;
     uint32_t *mask = nullptr;
     uint32_t *cand_count = nullptr, *cand_val = nullptr, *cand_idx = nullptr, *batch_seg = nullptr;
+    // power iteration support: per-item partial sums, per-layer coefficients and norms
+    double *pw_part = nullptr;
+    float *pw_coef = nullptr, *pw_norm = nullptr;
     // host-tensor staging (ta_step_host)
     float *st_w = nullptr, *st_hz = nullptr;
     void *st_g = nullptr;
@@ -97,7 +100,7 @@ template <typename T> cudaError_t dev_alloc(T **p, size_t count)
 
 void free_all(DeviceBuffers &d)
 {
-    void *ptrs[] = {d.verdict, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
+    void *ptrs[] = {d.pw_part, d.pw_coef, d.pw_norm, d.verdict, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
                     d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
     for (void *p : ptrs)
@@ -702,6 +705,54 @@ int ta_step_host(ta_handle *h, float *w_host, const void *g_host, const float *H
         }
         TA_CUDA(h, cudaStreamSynchronize(s));
     }
+    return TA_OK;
+}
+
+int ta_power_iterate(ta_handle *h, const float *u, const float *Hu, const float *V, const float *lambda_V, uint32_t m,
+                     float *u_next, float *lambda_out, float *norm_out, void *stream)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!u || !Hu || !u_next || !lambda_out) return fail(h, TA_ERR_ARG, "ta_power_iterate: u, Hu, u_next and lambda_out must not be NULL");
+    if (m > (uint32_t)ta::kMaxEigs) return fail(h, TA_ERR_ARG, "ta_power_iterate: at most TA_MAX_EIGS deflated vectors");
+    if (m > 0 && (!V || !lambda_V)) return fail(h, TA_ERR_ARG, "ta_power_iterate: V and lambda_V are needed when m > 0");
+    if (!aligned16(u) || !aligned16(Hu) || !aligned16(V) || !aligned16(u_next))
+        return fail(h, TA_ERR_ALIGN, "ta_power_iterate: every flat device buffer must be 16-byte aligned");
+    DeviceBuffers &d = h->d;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!d.pw_part) {
+        TA_CUDA(h, dev_alloc(&d.pw_part, (size_t)ta::kMaxEigs * h->n_items));
+        TA_CUDA(h, dev_alloc(&d.pw_coef, (size_t)ta::kMaxEigs * h->L));
+        TA_CUDA(h, dev_alloc(&d.pw_norm, h->L));
+    }
+    float *norm = norm_out ? norm_out : d.pw_norm;
+    ta::PowerArgs pa{d.items, h->n_items, h->n_batches, u, Hu, V, h->n_total, m, h->L, d.pw_part, d.pw_coef, norm, u_next};
+    ta::PowerLayerArgs la{d.item_lo, h->n_items, m, h->L, d.pw_part, lambda_V, d.pw_coef, lambda_out, norm};
+    const int grid = grid_for(h);
+    if (m > 0) {
+        ta::k_power<0><<<grid, ta::kThreads, 0, s>>>(pa);
+        ta::k_power_layer<0><<<h->L, ta::kThreads, 0, s>>>(la);
+        h->launches += 2;
+    }
+    ta::k_power<1><<<grid, ta::kThreads, 0, s>>>(pa);
+    ta::k_power_layer<1><<<h->L, ta::kThreads, 0, s>>>(la);
+    ta::k_power<2><<<grid, ta::kThreads, 0, s>>>(pa);
+    h->launches += 3;
+    TA_CUDA(h, cudaGetLastError());
+    h->last_stream = s;
+    return TA_OK;
+}
+
+int ta_set_curvature(ta_handle *h, const float *lambda_max_host)
+{
+    if (!h || !lambda_max_host) return TA_ERR_ARG;
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    std::vector<ta::LayerState> st(h->L);
+    TA_CUDA(h, cudaMemcpy(st.data(), h->d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost));
+    for (uint32_t l = 0; l < h->L; ++l) {
+        if (!(lambda_max_host[l] >= 0.f)) return fail(h, TA_ERR_ARG, "ta_set_curvature: values must be finite and >= 0");
+        st[l].lambda_max = lambda_max_host[l];
+    }
+    TA_CUDA(h, cudaMemcpy(h->d.state, st.data(), h->L * sizeof(ta::LayerState), cudaMemcpyHostToDevice));
     return TA_OK;
 }
 

@@ -195,3 +195,66 @@ def test_mask_dense_is_all_ones_and_gaps_stay_zero():
         assert ly.topk_threshold == np.float32(4) * a.min()          # k-th largest of |S| = P*a
         assert ly.lambda_max == a.max()                              # max|S| / P
     assert np.array_equal(_bits(mask, 0, n_total).astype(bool), inside)
+
+
+# ---------------------------------------------------------------- power iteration (Sec. 3.2)
+
+def _sym_blocks(sizes, seed):
+    rng = np.random.default_rng(seed)
+    table, off, mats = [], 3, []
+    for n in sizes:
+        A = rng.standard_normal((n, n))
+        # well separated spectrum so that a few dozen iterations converge
+        Q, _ = np.linalg.qr(A)
+        ev = np.concatenate([[10.0, -7.0, 4.0], rng.uniform(-1, 1, max(0, n - 3))])[:n]
+        mats.append((Q * ev) @ Q.T)
+        table.append((off, n))
+        off += n + 5
+    return table, (off + 7) // 8 * 8, mats
+
+
+def _apply(table, mats, u):
+    hu = np.zeros_like(u)
+    for (off, n), H in zip(table, mats):
+        hu[off:off + n] = (H @ u[off:off + n].astype(np.float64)).astype(np.float32)
+    return hu
+
+
+def test_power_iteration_finds_top_eigenvalues_with_deflation():
+    table, n_total, mats = _sym_blocks([6, 17, 40], seed=1)
+    rng = np.random.default_rng(2)
+    L = len(table)
+    found_v, found_lam = [], []
+    for k in range(3):                                   # top-3 by magnitude, one after the other
+        u = rng.standard_normal(n_total).astype(np.float32)
+        v = np.stack(found_v) if found_v else None
+        lam_v = np.stack(found_lam) if found_lam else None
+        for _ in range(200):
+            u, lam, nrm = orc.power_iterate(table, n_total, u, _apply(table, mats, u), v, lam_v)
+        found_v.append(u.copy())
+        found_lam.append(lam.copy())
+        for l, ((off, n), H) in enumerate(zip(table, mats)):
+            ev = np.linalg.eigvalsh(H)
+            want = sorted(ev, key=abs, reverse=True)[k]
+            assert lam[l] == pytest.approx(want, rel=1e-4), (k, l)
+            assert np.linalg.norm(u[off:off + n]) == pytest.approx(1.0, rel=1e-5)
+            assert nrm[l] == pytest.approx(abs(want), rel=1e-3)
+
+
+def test_power_iteration_rayleigh_quotient_closed_form():
+    # an exact eigenvector gives its eigenvalue; H = diag(d) and u = e_i make every quantity exact
+    n = 16
+    d = np.arange(1, n + 1, dtype=np.float32)
+    u = np.zeros(n, dtype=np.float32); u[4] = 2.0
+    out, lam, nrm = orc.power_iterate([(0, n)], n, u, d * u)
+    assert lam[0] == 5.0 and nrm[0] == 10.0 and out[4] == 1.0 and np.count_nonzero(out) == 1
+    # general u: float64 recomputation
+    rng = np.random.default_rng(0)
+    u = rng.standard_normal(n).astype(np.float32)
+    hu = (d * u).astype(np.float32)
+    out, lam, nrm = orc.power_iterate([(0, n)], n, u, hu)
+    assert lam[0] == pytest.approx(float((u.astype(np.float64) * hu).sum() / (u.astype(np.float64) ** 2).sum()), rel=1e-6)
+    assert np.allclose(out, hu / np.linalg.norm(hu.astype(np.float64)), rtol=1e-6)
+    # zero vector: defined as zeros
+    out, lam, nrm = orc.power_iterate([(0, n)], n, np.zeros(n, dtype=np.float32), np.zeros(n, dtype=np.float32))
+    assert lam[0] == 0.0 and nrm[0] == 0.0 and not out.any()
