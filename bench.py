@@ -318,6 +318,50 @@ def run_ours(args):
     return 0
 
 
+def run_power(args):
+    """Times ta_power_iterate (Sec. 3.2 support sweeps) on the workload's layer table; one JSON line."""
+    import torch
+    import paper_2508_16905_b200 as ta
+    from paper_2508_16905_b200 import workloads as W
+    torch.cuda.set_device(0)
+    wl = W.get(args.config)
+    N, L, m = wl.n_total, len(wl.table), args.deflate
+    h = ta.ta_create(wl.table, N, **wl.hparams())
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    u = torch.randn(N, generator=gen, device="cuda")
+    hu = torch.randn(N, generator=gen, device="cuda")
+    V = torch.randn(max(m, 1) * N, generator=gen, device="cuda") if m else None
+    lam_v = torch.rand(max(m, 1) * L, generator=gen, device="cuda") if m else None
+    out, lam = torch.empty(N, device="cuda"), torch.empty(L, device="cuda")
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    flush = torch.empty(64 << 20, dtype=torch.float32, device="cuda")       # 256 MB > L2, written between iterations
+    for _ in range(warmup):
+        ta.ta_power_iterate(h, u, hu, V, lam_v, m, out, lam)
+    times = []
+    for _ in range(steps):
+        flush.fill_(1.0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ta.ta_power_iterate(h, u, hu, V, lam_v, m, out, lam)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = sum(times) / len(times)
+    # algorithmic bytes: projections read u and m vectors; dots read u, Hu and m vectors; the write pass reads Hu and
+    # m vectors and writes u_next
+    bytes_alg = wl.num_params * 4 * ((1 + m if m else 0) + (2 + m) + (1 + m) + 1)
+    peak, kind = measured_peak()
+    print(json.dumps({"metric": "power-iteration step params/sec", "value": wl.num_params / (ms * 1e-3), "unit": UNIT,
+                      "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": wl.name, "params": wl.num_params, "layers": L, "deflated_vectors": m,
+                                 "l2": "256 MB written between iterations"},
+                      "roofline": {"bound": "hbm", "achieved": bytes_alg / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                                   "frac": bytes_alg / (ms * 1e-3) / 1e9 / peak, "peak_kind": kind, "traffic": None,
+                                   "algorithmic_bytes": bytes_alg}}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -328,7 +372,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--op", default="step", choices=["step", "power"], help="step: the optimizer pass (default); power: ta_power_iterate")
+    ap.add_argument("--deflate", type=int, default=0, help="--op power: number of deflated eigenvectors")
     args = ap.parse_args()
+    if args.op == "power":
+        return run_power(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)
