@@ -1,0 +1,64 @@
+"""Size limits and odd tables on the GPU: index arithmetic beyond 2^31, thousands of tiny layers."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2508_16905_b200 as ta
+from oracle import oracle as orc
+from tests.parity import ParityRun, oracle_hz
+
+pytestmark = pytest.mark.gpu
+
+
+def test_layer_longer_than_two_to_the_31():
+    # one layer of 2^31 + 4099 elements behind a small one: every flat index above 2^31 must be reached once.
+    # Checked through closed forms (the oracle would need minutes): g = +a on even, -a on odd flat indices.
+    n_big = (1 << 31) + 4099
+    table = [(8, 1000), (1016, n_big)]
+    n_total = (1016 + n_big + 7) // 8 * 8
+    a = 2.0 ** -10
+    h = ta.ta_create(table, n_total, beta=0.0, tau_low=1.0, tau_high=2.0, tau_curv=10.0, alpha=0.0, eta0=0.5)   # everything FP16
+    w = torch.zeros(n_total, device="cuda")
+    g = torch.empty(n_total, device="cuda")
+    g[0::2] = a
+    g[1::2] = -a
+    c = torch.full((n_total,), 0x5A5A, dtype=torch.int16, device="cuda")
+    hz = torch.ones(n_total, device="cuda")
+    hz[n_total - 9] = 3.0                                  # the layer's largest |S| sits in its last vector
+    ta.ta_step(h, w, g, hz, c, 0, 1)
+    stats, status = ta.ta_stats(h)
+    assert status.skipped == 0
+    s = stats[1]
+    mean = (a / n_big) if n_big % 2 else 0.0               # odd count: one unpaired element (the layer starts on an even index: +a)
+    assert s.grad_mean == pytest.approx(mean, abs=1e-12)
+    assert s.grad_var == pytest.approx(a * a - mean * mean, rel=1e-6)
+    assert s.lambda_max == 3.0 and s.topk_threshold == 1.0 and s.code == ta.TA_CODE_FP16
+    # w = -eta * g exactly; check the head, the tail beyond 2^31 and the gap
+    for lo, hi in [(1016, 1016 + 4096), (n_total - 8192, 1016 + n_big)]:
+        assert torch.equal(w[lo:hi], -0.5 * g[lo:hi])
+        want = (-0.5 * g[lo:hi]).to(torch.float16).view(torch.int16)
+        assert torch.equal(c[lo:hi], want)
+    assert float(w[1008:1016].abs().max()) == 0.0 and bool((c[1008:1016] == 0x5A5A).all())
+    assert float(w[1016 + n_big:].abs().max()) == 0.0
+    # every element was updated exactly once: the sum of |w| is n * eta * a (exact in float64)
+    total = float(w[1016:1016 + n_big].abs().sum(dtype=torch.float64))
+    assert total == pytest.approx(n_big * 0.5 * a, rel=1e-12)
+
+
+@pytest.mark.parametrize("ppm,P", [(1000000, 1), (300000, 2)])
+def test_thousands_of_tiny_layers(ppm, P):
+    # more layers than the one-launch path keeps in shared memory: the three-kernel path with a ragged table
+    rng = np.random.default_rng(P)
+    lengths = rng.integers(1, 40, 6000).tolist() + [5000, 70000]
+    table, off = [], 1
+    for j, n in enumerate(lengths):
+        off += int(j % 3 == 0)
+        table.append((off, int(n)))
+        off += int(n)
+    n_total = (off + 7) // 4 * 4
+    hp = dict(beta=0.5, tau_low=3e-7, tau_high=3e-6, tau_curv=0.5, topk_ppm=ppm, num_probes=P)
+    run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
+    D = np.exp(rng.uniform(np.log(1e-3), 0.0, n_total)).astype(np.float32)
+    for t in (1, 2):
+        g = torch.from_numpy((rng.standard_normal(n_total) * 1e-3).astype(np.float32)).cuda()
+        run.step(t, g, oracle_hz(D, P, 5, t), 5)
