@@ -192,7 +192,8 @@ def run_ours(args):
     state_bytes = N * 6
     # rotate over R buffer sets so that consecutive steps never find their inputs in L2
     R = 1 if (bytes_in_per_set + state_bytes) > 4 * l2_bytes else max(2, -(-6 * l2_bytes // (bytes_in_per_set + state_bytes)))
-    h = ta.ta_create(wl.table, N, **wl.hparams())
+    hp = dict(wl.hparams(), momentum=args.momentum, weight_decay=args.weight_decay)
+    h = ta.ta_create(wl.table, N, **hp)
     curv = W.make_curvature(wl, dev)
     sets = []
     z = torch.empty(N, device=dev)
@@ -249,7 +250,7 @@ def run_ours(args):
         e2e_steps = max(1, min(steps, args.e2e_steps))
         w_d, g_d, hz_d, c_d = sets[0]
         wh, gh, hzh, ch = (x.cpu().pin_memory() for x in (w_d, g_d, hz_d, c_d))
-        h2 = ta.ta_create(wl.table, N, **wl.hparams())
+        h2 = ta.ta_create(wl.table, N, **hp)
         ta.ta_step_host(h2, wh, gh, hzh, ch, wl.probe_seed, 1)          # warm-up: allocates the staging buffers
         torch.cuda.synchronize()
         D.barrier()
@@ -277,10 +278,11 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     g_b = 2 if wl.grad_dtype == "bf16" else 4
     copy_params = sum(n for (_, n), cd in zip(wl.table, codes) if cd < 2)
-    update_bytes = wl.num_params * (4 + g_b + 4) + 2 * copy_params
+    mom_b = 8 if args.momentum else 0          # momentum buffer read + write
+    update_bytes = wl.num_params * (4 + g_b + 4 + mom_b) + 2 * copy_params
     sweep_bytes = wl.num_params * (g_b + 4 * P)
     fused = ms_update < 1e-9          # small dense models run as one cooperative launch (k_fused)
-    step_bytes_min = wl.num_params * (4 + g_b + 4 * P + 4) + 2 * copy_params + (wl.num_params / 8 if wl.topk_ppm < 1000000 else 0)
+    step_bytes_min = wl.num_params * (4 + g_b + 4 * P + 4 + mom_b) + 2 * copy_params + (wl.num_params / 8 if wl.topk_ppm < 1000000 else 0)
     ms_step = ms / steps
     if fused:
         update_bytes, upd_ms = step_bytes_min, ms_step        # one kernel per step: its duration is the step time
@@ -307,7 +309,7 @@ def run_ours(args):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "params": wl.num_params, "layers": len(wl.table), "grad_dtype": wl.grad_dtype,
-                       "num_probes": P, "topk_ppm": wl.topk_ppm, "parallelism": f"replicas x{world}",
+                       "num_probes": P, "topk_ppm": wl.topk_ppm, "momentum": args.momentum, "weight_decay": args.weight_decay, "parallelism": f"replicas x{world}",
                        "l2": (f"inputs of one step ({(bytes_in_per_set + state_bytes) / 1e6:.0f} MB) exceed L2 ({l2_bytes / 1e6:.0f} MB)"
                               if R == 1 else f"{R} rotating buffer sets ({R * (bytes_in_per_set + state_bytes) / 1e6:.0f} MB) exceed L2 ({l2_bytes / 1e6:.0f} MB)"),
                        "codes": {"fp16": codes.count(0), "bf16": codes.count(1), "fp32": codes.count(2)}},
@@ -372,6 +374,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--momentum", type=float, default=0.0)
+    ap.add_argument("--weight-decay", type=float, default=0.0)
     ap.add_argument("--op", default="step", choices=["step", "power"], help="step: the optimizer pass (default); power: ta_power_iterate")
     ap.add_argument("--deflate", type=int, default=0, help="--op power: number of deflated eigenvectors")
     args = ap.parse_args()

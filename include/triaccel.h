@@ -78,8 +78,8 @@ typedef struct {
     uint32_t num_probes; /* P, one of 1, 2, 4, 8 */
     uint32_t t_ctrl;     /* decisions are taken at steps with step % t_ctrl == 0   Sec. 3.4 */
     uint32_t grad_dtype; /* TA_GRAD_F32 or TA_GRAD_BF16 */
-    float momentum;      /* must be 0 (plain SGD update) */
-    float weight_decay;  /* must be 0 */
+    float momentum;      /* SGD momentum mu in [0,1); 0 = plain SGD               Sec. 4.1 */
+    float weight_decay;  /* L2 coefficient wd >= 0 added to the gradient; 0 = none       */
     uint32_t flags;      /* must be 0 */
 } ta_hparams;
 
@@ -125,7 +125,10 @@ int ta_destroy(ta_handle *h);
 /*
  * ta_step -- one optimizer pass (asynchronous).
  *   w      device float[n_total], FP32 master weights, updated in place:
- *          w_i <- fl32(w_i - eta_l * g_i), eta_l = fl32(eta0 * s_l)                  (Sec. 3.2, 4.1)
+ *          w_i <- fl32(w_i - eta_l * b_i), eta_l = fl32(eta0 * s_l)                  (Sec. 3.2, 4.1)
+ *          with b_i = g_i for plain SGD; with weight decay d_i = fl32(g_i + wd * w_i); with momentum
+ *          b_i <- fl32(mu * b_i + d_i) in a library-owned buffer that starts at zero (no dampening,
+ *          no Nesterov step: the rule of the paper's SGD baselines)
  *   g      device, float[n_total] or bfloat16[n_total] per hp.grad_dtype; read only
  *   Hz     device float[P][n_total] (probe p at Hz + p * n_total), the caller's products
  *          H z^(p) with z^(p) = the probe ta_probe() writes for (probe_seed, step, p); or NULL,

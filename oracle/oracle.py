@@ -22,7 +22,7 @@ class HParams(C.Structure):
     _fields_ = [("beta", C.c_float), ("tau_low", C.c_float), ("tau_high", C.c_float),
                 ("tau_curv", C.c_float), ("alpha", C.c_float), ("eta0", C.c_float),
                 ("topk_ppm", C.c_uint32), ("num_probes", C.c_uint32), ("t_ctrl", C.c_uint32),
-                ("grad_dtype", C.c_uint32)]
+                ("grad_dtype", C.c_uint32), ("momentum", C.c_float), ("weight_decay", C.c_float)]
 
 
 class Layer(C.Structure):
@@ -53,6 +53,7 @@ def lib():
         L.orc_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64]
         L.orc_get_layers.argtypes = [C.c_void_p, C.POINTER(Layer)]
         L.orc_get_status.argtypes = [C.c_void_p, C.POINTER(Status)]
+        L.orc_get_momentum.argtypes = [C.c_void_p, C.c_void_p]
         L.orc_get_mask.argtypes = [C.c_void_p, C.c_void_p]
         L.orc_mask_words.restype = C.c_uint64
         L.orc_mask_words.argtypes = [C.c_void_p]
@@ -148,12 +149,12 @@ class Oracle:
     """Per-layer optimizer state plus the step, on the host."""
 
     def __init__(self, table, n_total, beta=0.9, tau_low=1e-7, tau_high=1e-5, tau_curv=0.9, alpha=1.0,
-                 eta0=0.1, topk_ppm=1000000, num_probes=1, t_ctrl=1, grad_dtype="f32"):
+                 eta0=0.1, topk_ppm=1000000, num_probes=1, t_ctrl=1, grad_dtype="f32", momentum=0.0, weight_decay=0.0):
         self.L = len(table)
         self.n_total = int(n_total)
         segs = (Segment * self.L)(*[Segment(int(o), int(n)) for o, n in table])
         self.hp = HParams(beta, tau_low, tau_high, tau_curv, alpha, eta0, topk_ppm, num_probes, t_ctrl,
-                          1 if grad_dtype == "bf16" else 0)
+                          1 if grad_dtype == "bf16" else 0, momentum, weight_decay)
         self.grad_bf16 = grad_dtype == "bf16"
         self._h = lib().orc_create(segs, self.L, self.n_total, C.byref(self.hp))
         if not self._h:
@@ -191,6 +192,11 @@ class Oracle:
         n = lib().orc_mask_words(self._h)
         m = np.zeros(n, dtype=np.uint32)
         lib().orc_get_mask(self._h, _ptr(m))
+        return m
+
+    def momentum_buffer(self):
+        m = np.zeros(self.n_total, dtype=np.float32)
+        lib().orc_get_momentum(self._h, _ptr(m))
         return m
 
     def codes(self):

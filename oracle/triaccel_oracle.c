@@ -51,6 +51,8 @@ typedef struct {
     uint32_t num_probes;  /* P */
     uint32_t t_ctrl;      /* control interval, >= 1 */
     uint32_t grad_dtype;  /* 0 = float, 1 = bfloat16 */
+    float momentum;       /* SGD momentum (Sec. 4.1 names 0.9 for the baselines); 0 = none */
+    float weight_decay;   /* L2 coefficient added to the gradient; 0 = none */
 } orc_hparams;
 
 typedef struct {
@@ -81,6 +83,7 @@ typedef struct {
     orc_layer *layer;
     uint32_t *mask;       /* one bit per flat element, bit (i & 31) of word i >> 5 */
     uint64_t mask_words;
+    float *mom;           /* momentum buffer, one float per flat element, starts at zero */
     orc_status status;
 } orc_state;
 
@@ -235,18 +238,20 @@ orc_state *orc_create(const orc_segment *table, uint32_t L, uint64_t n_total, co
     }
     st->mask_words = (n_total + 31u) / 32u;
     st->mask = (uint32_t *)calloc(st->mask_words ? st->mask_words : 1, sizeof(uint32_t));
+    st->mom = hp->momentum != 0.0f ? (float *)calloc(n_total ? n_total : 1, sizeof(float)) : NULL;
     return st;
 }
 
 void orc_destroy(orc_state *st)
 {
     if (!st) return;
-    free(st->seg); free(st->layer); free(st->mask); free(st);
+    free(st->seg); free(st->layer); free(st->mask); free(st->mom); free(st);
 }
 
 void orc_set_lr(orc_state *st, float eta0) { st->hp.eta0 = eta0; }
 void orc_get_layers(const orc_state *st, orc_layer *out) { memcpy(out, st->layer, sizeof(orc_layer) * st->L); }
 void orc_get_status(const orc_state *st, orc_status *out) { *out = st->status; }
+void orc_get_momentum(const orc_state *st, float *out) { if (st->mom) memcpy(out, st->mom, sizeof(float) * st->n_total); }
 void orc_get_mask(const orc_state *st, uint32_t *out) { memcpy(out, st->mask, sizeof(uint32_t) * st->mask_words); }
 uint64_t orc_mask_words(const orc_state *st) { return st->mask_words; }
 uint64_t orc_sizeof_layer(void) { return sizeof(orc_layer); }
@@ -423,7 +428,12 @@ int orc_step(orc_state *st, float *w, const void *g_any, const float *hz, uint16
         /* step 7: master update and cast (Sec. 2 master copy; Sec. 3.2; Sec. 4.1 SGD) */
         for (uint64_t j = 0; j < n; ++j) {
             uint64_t i = off + j;
-            float wn = (float)((double)w[i] - eta * (double)gl[j]);
+            /* SGD with weight decay and momentum (Sec. 4.1): d = g + wd w; b = mu b + d; w = w - eta b.
+             * d and b are float, one rounding each (fused multiply-add); the buffer starts at zero. */
+            float dir = gl[j];
+            if (hp->weight_decay != 0.0f) dir = fmaf(hp->weight_decay, w[i], dir);
+            if (st->mom) { dir = fmaf(hp->momentum, st->mom[i], dir); st->mom[i] = dir; }
+            float wn = (float)((double)w[i] - eta * (double)dir);
             w[i] = wn;
             if (ly->code == 0u) c[i] = orc_f32_to_f16(wn);
             else if (ly->code == 1u) c[i] = orc_f32_to_bf16(wn);

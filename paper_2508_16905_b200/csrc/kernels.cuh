@@ -663,7 +663,18 @@ struct ApplyArgs {
     uint16_t *c;
     const LayerState *state;
     const Status *status;
+    float *mom;                  // momentum buffer [n_total] or NULL
+    float momentum, weight_decay;
 };
+
+// Direction of the SGD update (Sec. 4.1): d = g + wd w, then b = mu b + d with the buffer updated in place.
+// One float rounding each.
+__device__ __forceinline__ float sgd_direction(float g, float w, float *buf, float momentum, float weight_decay)
+{
+    float d = weight_decay != 0.f ? fmaf(weight_decay, w, g) : g;
+    if (buf) { d = fmaf(momentum, *buf, d); *buf = d; }
+    return d;
+}
 
 __device__ __forceinline__ uint16_t cast16(float x, uint32_t code)
 {
@@ -693,13 +704,23 @@ __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, 
             for (uint32_t e = 0; e < 4; ++e) {
                 const uint64_t i = i0 + e;
                 if (i >= begin && i < end) {
-                    const float wn = fmaf(neg_eta, GradVec<BF16>::load1(A.g, i), A.w[i]);
+                    const float w_old = A.w[i];
+                    const float dir = sgd_direction(GradVec<BF16>::load1(A.g, i), w_old, A.mom ? A.mom + i : nullptr, A.momentum, A.weight_decay);
+                    const float wn = fmaf(neg_eta, dir, w_old);
                     A.w[i] = wn;
                     if (code < 2u) A.c[i] = cast16(wn, code);
                 }
             }
         };
         auto store_row = [&](uint64_t i0, float4 wv, float4 gv) {
+            if (A.mom || A.weight_decay != 0.f) {      // uniform over the launch
+                float4 mv = A.mom ? __ldcs(reinterpret_cast<const float4 *>(A.mom + i0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                gv.x = sgd_direction(gv.x, wv.x, A.mom ? &mv.x : nullptr, A.momentum, A.weight_decay);
+                gv.y = sgd_direction(gv.y, wv.y, A.mom ? &mv.y : nullptr, A.momentum, A.weight_decay);
+                gv.z = sgd_direction(gv.z, wv.z, A.mom ? &mv.z : nullptr, A.momentum, A.weight_decay);
+                gv.w = sgd_direction(gv.w, wv.w, A.mom ? &mv.w : nullptr, A.momentum, A.weight_decay);
+                if (A.mom) *reinterpret_cast<float4 *>(A.mom + i0) = mv;
+            }
             wv.x = fmaf(neg_eta, gv.x, wv.x);
             wv.y = fmaf(neg_eta, gv.y, wv.y);
             wv.z = fmaf(neg_eta, gv.z, wv.z);

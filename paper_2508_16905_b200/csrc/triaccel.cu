@@ -35,6 +35,7 @@ struct DeviceBuffers {
     double *pw_part = nullptr;
     float *pw_coef = nullptr, *pw_norm = nullptr;
     // host-tensor staging (ta_step_host)
+    float *mom = nullptr;                         // SGD momentum buffer [n_total], only when momentum != 0
     float *st_w = nullptr, *st_hz = nullptr;
     void *st_g = nullptr;
     uint16_t *st_c = nullptr;
@@ -100,7 +101,7 @@ template <typename T> cudaError_t dev_alloc(T **p, size_t count)
 
 void free_all(DeviceBuffers &d)
 {
-    void *ptrs[] = {d.pw_part, d.pw_coef, d.pw_norm, d.verdict, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
+    void *ptrs[] = {d.mom, d.pw_part, d.pw_coef, d.pw_norm, d.verdict, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
                     d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
     for (void *p : ptrs)
@@ -168,7 +169,8 @@ void launch_apply(ta_handle *h, float *w, const void *g, uint16_t *c, uint32_t i
 {
     if (item_count == 0) return;
     const uint32_t batches = (item_count + ta::kWarps - 1) / ta::kWarps;
-    ta::ApplyArgs aa{h->d.items + item_begin, item_count, batches, w, g, c, h->d.state, h->d.status};
+    ta::ApplyArgs aa{h->d.items + item_begin, item_count, batches, w, g, c, h->d.state, h->d.status,
+                     h->d.mom, h->hp.momentum, h->hp.weight_decay};
     const int grid = (int)std::min<long long>(batches, (long long)h->sm_count * 8);
     if (h->hp.grad_dtype == TA_GRAD_BF16) ta::k_apply<true><<<grid, ta::kThreads, 0, s>>>(aa);
     else ta::k_apply<false><<<grid, ta::kThreads, 0, s>>>(aa);
@@ -248,8 +250,9 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     if (hp->topk_ppm == 0 || hp->topk_ppm > 1000000u) return fail(nullptr, TA_ERR_ARG, "ta_create: topk_ppm must be in [1, 1000000]");
     if (hp->t_ctrl == 0) return fail(nullptr, TA_ERR_ARG, "ta_create: t_ctrl must be >= 1");
     if (hp->grad_dtype != TA_GRAD_F32 && hp->grad_dtype != TA_GRAD_BF16) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown grad_dtype");
-    if (hp->momentum != 0.f || hp->weight_decay != 0.f || hp->flags != 0u)
-        return fail(nullptr, TA_ERR_ARG, "ta_create: momentum, weight_decay and flags must be 0");
+    if (!(hp->momentum >= 0.f && hp->momentum < 1.f)) return fail(nullptr, TA_ERR_ARG, "ta_create: momentum must be in [0,1)");
+    if (!(hp->weight_decay >= 0.f) || !(hp->weight_decay < 1e30f)) return fail(nullptr, TA_ERR_ARG, "ta_create: weight_decay must be finite and >= 0");
+    if (hp->flags != 0u) return fail(nullptr, TA_ERR_ARG, "ta_create: flags must be 0");
     if (n_total % 4 != 0) return fail(nullptr, TA_ERR_ARG, "ta_create: n_total must be a multiple of 4");
     uint64_t end = 0, n_params = 0;
     for (uint32_t l = 0; l < L; ++l) {
@@ -302,7 +305,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         int coop = 0;
         TA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device));
         const size_t smem = (size_t)L * 8;
-        if (coop && !h->topk && n_params <= fused_max_params() && smem <= 32 * 1024) {
+        if (coop && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f && n_params <= fused_max_params() && smem <= 32 * 1024) {
             const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
             h->fused_ok = true;
             fused_blocks = 1ll << 40;
@@ -419,6 +422,10 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     TA_TRY(cudaMemcpy(d.state, init.data(), L * sizeof(ta::LayerState), cudaMemcpyHostToDevice));
     TA_TRY(cudaMemset(d.scratch, 0, L * sizeof(ta::LayerScratch)));
     TA_TRY(cudaMemset(d.status, 0, sizeof(ta::Status)));
+    if (hp->momentum != 0.f) {
+        TA_TRY(dev_alloc(&d.mom, n_total));
+        TA_TRY(cudaMemset(d.mom, 0, n_total * sizeof(float)));
+    }
     if (h->fused_ok) {
         TA_TRY(dev_alloc(&d.verdict, L));
         TA_TRY(dev_alloc(&d.barrier, 1));
@@ -532,7 +539,7 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
         fa.sweep.g = g; fa.sweep.hz = Hz; fa.sweep.n_total = h->n_total; fa.sweep.seed = probe_seed; fa.sweep.step = (uint32_t)step;
         fa.sweep.p_s1 = d.p_s1; fa.sweep.p_s2 = d.p_s2; fa.sweep.p_sa = d.p_sa;
         fa.sweep.p_amax = d.p_amax; fa.sweep.p_amin = d.p_amin; fa.sweep.p_bad = d.p_bad;
-        fa.apply = ta::ApplyArgs{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status};
+        fa.apply = ta::ApplyArgs{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status, nullptr, 0.f, 0.f};
         fa.item_lo = d.item_lo; fa.seg_len = d.seg_len; fa.verdict = d.verdict;
         fa.state = d.state; fa.status = d.status;
         fa.dp.hp = hyper_of(h->hp); fa.dp.eta0 = h->hp.eta0; fa.dp.has_hz = Hz ? 1u : 0u;
@@ -826,7 +833,8 @@ int ta_masks(ta_handle *h, const uint32_t **dev_bits, uint64_t *num_words)
 int ta_state_size(ta_handle *h, uint64_t *bytes)
 {
     if (!h || !bytes) return TA_ERR_ARG;
-    *bytes = sizeof(StateHeader) + h->L * sizeof(ta::LayerState) + sizeof(ta::Status) + h->mask_words * sizeof(uint32_t);
+    *bytes = sizeof(StateHeader) + h->L * sizeof(ta::LayerState) + sizeof(ta::Status) + h->mask_words * sizeof(uint32_t) +
+             (h->d.mom ? h->n_total * sizeof(float) : 0);
     return TA_OK;
 }
 
@@ -848,6 +856,8 @@ int ta_state_save(ta_handle *h, void *buf_host, uint64_t bytes)
     TA_CUDA(h, cudaMemcpy(p, h->d.status, sizeof(ta::Status), cudaMemcpyDeviceToHost));
     p += sizeof(ta::Status);
     if (h->mask_words) TA_CUDA(h, cudaMemcpy(p, h->d.mask, h->mask_words * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    p += h->mask_words * sizeof(uint32_t);
+    if (h->d.mom) TA_CUDA(h, cudaMemcpy(p, h->d.mom, h->n_total * sizeof(float), cudaMemcpyDeviceToHost));
     return TA_OK;
 }
 
@@ -872,6 +882,8 @@ int ta_state_load(ta_handle *h, const void *buf_host, uint64_t bytes)
     TA_CUDA(h, cudaMemcpy(h->d.status, p, sizeof(ta::Status), cudaMemcpyHostToDevice));
     p += sizeof(ta::Status);
     if (h->mask_words) TA_CUDA(h, cudaMemcpy(h->d.mask, p, h->mask_words * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    p += h->mask_words * sizeof(uint32_t);
+    if (h->d.mom) TA_CUDA(h, cudaMemcpy(h->d.mom, p, h->n_total * sizeof(float), cudaMemcpyHostToDevice));
     h->hp.eta0 = hd.hp.eta0;
     h->last_step = hd.last_step;
     h->stepped = hd.stepped != 0;

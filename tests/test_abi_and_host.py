@@ -49,7 +49,9 @@ def test_create_rejects_bad_arguments_before_touching_a_device():
         dict(table=[(0, 8)], n_total=8, topk_ppm=0),
         dict(table=[(0, 8)], n_total=8, beta=1.0),
         dict(table=[(0, 8)], n_total=8, t_ctrl=0),
-        dict(table=[(0, 8)], n_total=8, momentum=0.9),
+        dict(table=[(0, 8)], n_total=8, momentum=1.0),
+        dict(table=[(0, 8)], n_total=8, weight_decay=-1.0),
+        dict(table=[(0, 8)], n_total=8, flags=1),
         dict(table=[(0, 8)], n_total=8, tau_low=2.0, tau_high=1.0),
     ]
     for kw in bad:

@@ -368,3 +368,38 @@ def test_bounded_wait_runs_out_without_hanging():
     ta.ta_step(hs[1], ws[1], g2, None, cs[1], 0, 3)
     assert torch.equal(ws[0].view(torch.int32), ws[1].view(torch.int32)) and torch.equal(cs[0], cs[1])
     assert ta.ta_stats(hs[0])[1].skipped == 0
+
+
+@pytest.mark.parametrize("momentum,wd,grad_dtype", [(0.9, 0.0, "f32"), (0.0, 5e-4, "f32"), (0.9, 5e-4, "bf16")])
+def test_momentum_and_weight_decay(momentum, wd, grad_dtype):
+    table, n_total = ragged_table(RAGGED)
+    rng = np.random.default_rng(11)
+    hp = dict(beta=0.5, tau_low=3e-7, tau_high=3e-6, eta0=0.05, momentum=momentum, weight_decay=wd, grad_dtype=grad_dtype)
+    run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
+    D = np.exp(rng.uniform(np.log(1e-4), 0.0, n_total)).astype(np.float32)
+    for t in range(1, 9):
+        g = torch.from_numpy((rng.standard_normal(n_total) * 1e-3).astype(np.float32)).cuda()
+        if grad_dtype == "bf16":
+            g = g.to(torch.bfloat16)
+        if t == 5:
+            g[table[3][0]] = float("inf")             # skipped: weights AND momentum buffer stay as they are
+        run.step(t, g, oracle_hz(D, 1, 2, t) if t % 2 else None, 2)
+
+
+def test_momentum_state_is_checkpointed():
+    wl = W.get("mlp_tiny")
+    hp = dict(wl.hparams(), momentum=0.9, weight_decay=1e-4)
+    a = ta.ta_create(wl.table, wl.n_total, **hp)
+    wa = W.make_weights(wl, "cuda")
+    ca = torch.zeros(wl.n_total, dtype=torch.int16, device="cuda")
+    for t in (1, 2, 3):
+        ta.ta_step(a, wa, W.make_grads(wl, t, "cuda"), None, ca, 0, t)
+    blob = ta.ta_state_save(a)
+    b = ta.ta_create(wl.table, wl.n_total, **hp)
+    ta.ta_state_load(b, blob)
+    wb, cb = wa.clone(), ca.clone()
+    for t in (4, 5):
+        g = W.make_grads(wl, t, "cuda")
+        ta.ta_step(a, wa, g, None, ca, 0, t)
+        ta.ta_step(b, wb, g, None, cb, 0, t)
+        assert torch.equal(wa.view(torch.int32), wb.view(torch.int32)) and torch.equal(ca, cb)

@@ -250,3 +250,39 @@ def test_batch_rule_truth_table():
     assert orc.batch_next(96, mem_usage=90.0, **args) == 96
     assert orc.batch_next(124, mem_usage=10.0, **args) == 128      # clamps
     assert orc.batch_next(16, mem_usage=99.0, **args) == 8
+
+
+# ---------------------------------------------------------------- momentum and weight decay (Sec. 4.1 SGD)
+
+@pytest.mark.parametrize("momentum,wd", [(0.9, 0.0), (0.0, 5e-4), (0.9, 5e-4)])
+def test_momentum_and_weight_decay_follow_torch_sgd(momentum, wd):
+    # an independent implementation of the same update rule: torch.optim.SGD (no dampening, no Nesterov)
+    n = 3000
+    rng = np.random.default_rng(0)
+    w0 = rng.standard_normal(n).astype(F)
+    o = orc.Oracle([(0, n)], n, alpha=0.0, eta0=0.05, momentum=momentum, weight_decay=wd, tau_low=-2.0, tau_high=-1.0)
+    w, c = w0.copy(), np.zeros(n, dtype=np.uint16)
+    p = torch.nn.Parameter(torch.from_numpy(w0.copy()))
+    opt = torch.optim.SGD([p], lr=0.05, momentum=momentum, weight_decay=wd)
+    for t in range(1, 9):
+        g = (rng.standard_normal(n) * 0.1).astype(F)
+        o.step(w, g, None, c, 0, t)
+        p.grad = torch.from_numpy(g.copy())
+        opt.step()
+        assert np.allclose(w, p.detach().numpy(), rtol=2e-6, atol=1e-7), t
+    if momentum:
+        buf = opt.state[p]["momentum_buffer"].numpy()
+        assert np.allclose(o.momentum_buffer(), buf, rtol=2e-6, atol=1e-6)
+
+
+def test_momentum_buffer_untouched_by_a_skipped_step():
+    n = 64
+    o = orc.Oracle([(0, n)], n, momentum=0.9)
+    w, c = np.ones(n, dtype=F), np.zeros(n, dtype=np.uint16)
+    g = np.full(n, 0.5, dtype=F)
+    o.step(w, g, None, c, 0, 1)
+    before = (w.copy(), o.momentum_buffer())
+    g2 = g.copy(); g2[3] = np.nan
+    assert o.step(w, g2, None, c, 0, 2) is True
+    assert np.array_equal(w, before[0]) and np.array_equal(o.momentum_buffer(), before[1])
+    assert np.all(before[1] == 0.5)
