@@ -28,6 +28,9 @@
 #ifndef TA_SWEEP_ROWS_P4
 #define TA_SWEEP_ROWS_P4 2
 #endif
+#ifndef TA_SWEEP_MIN_BLOCKS_P4
+#define TA_SWEEP_MIN_BLOCKS_P4 1
+#endif
 #ifndef TA_APPLY_ROWS
 #define TA_APPLY_ROWS 4
 #endif
@@ -228,7 +231,10 @@ template <int P> __device__ __forceinline__ float pairwise(const float (&t)[P > 
 
 template <int P, bool TOPK> struct SweepAcc {
     double s1 = 0.0, s2 = 0.0, sa = 0.0;
-    uint32_t amax = 0u, amin = 0xFFFFFFFFu, gmax = 0u, hmax = 0u;
+    float sa_row = 0.f;     // |S| of the current row (four values), folded into sa by end_row()
+    uint32_t amax = 0u, amin = 0xFFFFFFFFu, gmax = 0u;
+
+    __device__ __forceinline__ void end_row() { sa += (double)sa_row; sa_row = 0.f; }
 
     // one element: gradient value gv, probe products hv[p], sign words sel[p], bit position pos
     __device__ __forceinline__ uint32_t element(float gv, const float (&hv)[P > 0 ? P : 1],
@@ -247,7 +253,6 @@ template <int P, bool TOPK> struct SweepAcc {
 #pragma unroll
             for (int p = 0; p < P; ++p) {
                 const uint32_t hb = __float_as_uint(hv[p]);
-                hmax = max(hmax, hb & 0x7FFFFFFFu);
                 t[p] = __uint_as_float(hb ^ (((sel[p] >> pos) & 1u) << 31));
             }
             ab = __float_as_uint(pairwise<P>(t)) & 0x7FFFFFFFu;
@@ -255,7 +260,7 @@ template <int P, bool TOPK> struct SweepAcc {
         if (P > 0) {
             amax = max(amax, ab);
             amin = min(amin, ab);
-            if (TOPK) sa += (double)__uint_as_float(ab);
+            if (TOPK) sa_row += __uint_as_float(ab);
         }
         return ab;
     }
@@ -331,6 +336,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                     }
                 }
             }
+            if (TOPK) acc.end_row();
         };
 
         auto full_rows = [&](uint64_t row, RowData<P> (&rd)[U], int count) {
@@ -356,6 +362,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                         if (TOPK) hist_add(ab);
                     }
                     if (TOPK) {
+                        acc.end_row();
                         const uint64_t i0 = (row + u) * 128ull + lane * 4u;
                         *reinterpret_cast<float4 *>(A.abs_s + i0) = make_float4(av[0], av[1], av[2], av[3]);
                     }
@@ -412,7 +419,9 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
         const uint32_t amax = __reduce_max_sync(0xFFFFFFFFu, acc.amax);
         const uint32_t amin = __reduce_min_sync(0xFFFFFFFFu, acc.amin);
         const uint32_t gmax = __reduce_max_sync(0xFFFFFFFFu, acc.gmax);
-        const uint32_t hmax = __reduce_max_sync(0xFFFFFFFFu, P == 1 ? acc.amax : acc.hmax);
+        // a non-finite Hz value always makes its probe sum non-finite, so max|S| flags it (a sum of finite values
+        // that overflows also lands here; the exact recount below then finds nothing)
+        const uint32_t hmax = amax;
         uint32_t bad = 0;
         if (gmax >= kNonFiniteBits || (P > 0 && hmax >= kNonFiniteBits)) {
             // rare: count the non-finite inputs of this item exactly
@@ -444,7 +453,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
 }
 
 template <int P, bool BF16, bool TOPK>
-__global__ void __launch_bounds__(kThreads) k_sweep(const SweepArgs A)
+__global__ void __launch_bounds__(kThreads, (P >= 4 ? TA_SWEEP_MIN_BLOCKS_P4 : 1)) k_sweep(const SweepArgs A)
 {
     __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
     for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK>(A, batch, sh_hist);
