@@ -1016,48 +1016,67 @@ __global__ void __launch_bounds__(kThreads) k_power(const PowerArgs A)
             for (int j = 0; j < kMaxEigs; ++j) a[j] = (MODE != 0 && j < (int)A.m) ? A.coef[(uint64_t)j * A.L + item.seg] : 0.f;
             const float nrm = MODE == 2 ? A.norm[item.seg] : 1.f;
             const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
-            for (uint64_t row = row_first; row <= row_last; ++row) {
-                const uint64_t i0 = row * 128ull + lane * 4u;
-                const bool full = row * 128ull >= begin && row * 128ull + 128u <= end;
-                if (MODE == 0) {
-                    const float4 uu = load_row4(A.u, i0, full, begin, end);
+            constexpr int UR = 4;                          // rows whose loads are issued together
+            uint64_t row = row_first;
+            while (row <= row_last) {
+                const bool group = row * 128ull >= begin && (row + UR) * 128ull <= end;
+                const int cnt = group ? UR : 1;
+                const bool full = group || (row * 128ull >= begin && row * 128ull + 128u <= end);
+                float4 uu[UR], t[UR];
 #pragma unroll
-                    for (int j = 0; j < kMaxEigs; ++j) {
-                        if (j < (int)A.m) {
-                            const float4 vv = load_row4(A.v + (uint64_t)j * A.n_total, i0, full, begin, end);
-                            acc[j] += (double)vv.x * (double)uu.x + (double)vv.y * (double)uu.y +
-                                      (double)vv.z * (double)uu.z + (double)vv.w * (double)uu.w;
-                        }
+                for (int r = 0; r < UR; ++r) {
+                    if (r < cnt) {
+                        const uint64_t i0 = (row + r) * 128ull + lane * 4u;
+                        if (MODE != 2) uu[r] = load_row4(A.u, i0, full, begin, end);
+                        if (MODE != 0) t[r] = load_row4(A.hu, i0, full, begin, end);
                     }
-                } else {
-                    float4 t = load_row4(A.hu, i0, full, begin, end);
+                }
 #pragma unroll
-                    for (int j = 0; j < kMaxEigs; ++j) {
-                        if (j < (int)A.m) {
-                            const float4 vv = load_row4(A.v + (uint64_t)j * A.n_total, i0, full, begin, end);
-                            t.x = fmaf(-a[j], vv.x, t.x); t.y = fmaf(-a[j], vv.y, t.y);
-                            t.z = fmaf(-a[j], vv.z, t.z); t.w = fmaf(-a[j], vv.w, t.w);
-                        }
-                    }
-                    if (MODE == 1) {
-                        const float4 uu = load_row4(A.u, i0, full, begin, end);
-                        acc[0] += (double)uu.x * (double)uu.x + (double)uu.y * (double)uu.y + (double)uu.z * (double)uu.z + (double)uu.w * (double)uu.w;
-                        acc[1] += (double)uu.x * (double)t.x + (double)uu.y * (double)t.y + (double)uu.z * (double)t.z + (double)uu.w * (double)t.w;
-                        acc[2] += (double)t.x * (double)t.x + (double)t.y * (double)t.y + (double)t.z * (double)t.z + (double)t.w * (double)t.w;
-                    } else {
-                        float4 o;
-                        o.x = nrm > 0.f ? __fdiv_rn(t.x, nrm) : 0.f; o.y = nrm > 0.f ? __fdiv_rn(t.y, nrm) : 0.f;
-                        o.z = nrm > 0.f ? __fdiv_rn(t.z, nrm) : 0.f; o.w = nrm > 0.f ? __fdiv_rn(t.w, nrm) : 0.f;
-                        if (full) {
-                            *reinterpret_cast<float4 *>(A.u_next + i0) = o;
-                        } else {
-                            if (i0 + 0 >= begin && i0 + 0 < end) A.u_next[i0 + 0] = o.x;
-                            if (i0 + 1 >= begin && i0 + 1 < end) A.u_next[i0 + 1] = o.y;
-                            if (i0 + 2 >= begin && i0 + 2 < end) A.u_next[i0 + 2] = o.z;
-                            if (i0 + 3 >= begin && i0 + 3 < end) A.u_next[i0 + 3] = o.w;
+                for (int j = 0; j < kMaxEigs; ++j) {
+                    if (j < (int)A.m) {
+                        float4 vv[UR];
+#pragma unroll
+                        for (int r = 0; r < UR; ++r)
+                            if (r < cnt) vv[r] = load_row4(A.v + (uint64_t)j * A.n_total, (row + r) * 128ull + lane * 4u, full, begin, end);
+#pragma unroll
+                        for (int r = 0; r < UR; ++r) {
+                            if (r < cnt) {
+                                if (MODE == 0) {
+                                    acc[j] += (double)vv[r].x * (double)uu[r].x + (double)vv[r].y * (double)uu[r].y +
+                                              (double)vv[r].z * (double)uu[r].z + (double)vv[r].w * (double)uu[r].w;
+                                } else {
+                                    t[r].x = fmaf(-a[j], vv[r].x, t[r].x); t[r].y = fmaf(-a[j], vv[r].y, t[r].y);
+                                    t[r].z = fmaf(-a[j], vv[r].z, t[r].z); t[r].w = fmaf(-a[j], vv[r].w, t[r].w);
+                                }
+                            }
                         }
                     }
                 }
+#pragma unroll
+                for (int r = 0; r < UR; ++r) {
+                    if (r < cnt) {
+                        const uint64_t i0 = (row + r) * 128ull + lane * 4u;
+                        if (MODE == 1) {
+                            const float4 q = uu[r], p = t[r];
+                            acc[0] += (double)q.x * (double)q.x + (double)q.y * (double)q.y + (double)q.z * (double)q.z + (double)q.w * (double)q.w;
+                            acc[1] += (double)q.x * (double)p.x + (double)q.y * (double)p.y + (double)q.z * (double)p.z + (double)q.w * (double)p.w;
+                            acc[2] += (double)p.x * (double)p.x + (double)p.y * (double)p.y + (double)p.z * (double)p.z + (double)p.w * (double)p.w;
+                        } else if (MODE == 2) {
+                            float4 o;
+                            o.x = nrm > 0.f ? __fdiv_rn(t[r].x, nrm) : 0.f; o.y = nrm > 0.f ? __fdiv_rn(t[r].y, nrm) : 0.f;
+                            o.z = nrm > 0.f ? __fdiv_rn(t[r].z, nrm) : 0.f; o.w = nrm > 0.f ? __fdiv_rn(t[r].w, nrm) : 0.f;
+                            if (full) {
+                                *reinterpret_cast<float4 *>(A.u_next + i0) = o;
+                            } else {
+                                if (i0 + 0 >= begin && i0 + 0 < end) A.u_next[i0 + 0] = o.x;
+                                if (i0 + 1 >= begin && i0 + 1 < end) A.u_next[i0 + 1] = o.y;
+                                if (i0 + 2 >= begin && i0 + 2 < end) A.u_next[i0 + 2] = o.z;
+                                if (i0 + 3 >= begin && i0 + 3 < end) A.u_next[i0 + 3] = o.w;
+                            }
+                        }
+                    }
+                }
+                row += cnt;
             }
         }
         if (MODE != 2) {
