@@ -42,17 +42,19 @@ def kernel_source_hash():
     return h.hexdigest()[:16]
 
 
-def recorded_traffic(kernel, workload, units):
-    """DRAM bytes per launch of `kernel` from the committed ncu capture, or None when there is no
-    capture for this workload or the kernel source changed since it was taken."""
+def recorded_traffic(workload, units):
+    """(DRAM bytes per launch of the dominant kernel, DRAM bytes per step over all kernels) from the committed ncu
+    captures, or (None, None) when there is none for this workload or the kernel source changed since."""
     try:
         with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
-            rec = json.load(f)[kernel]
+            rec = json.load(f)
+        if rec.get("kernels_cuh_sha256_16") != kernel_source_hash():
+            return None, None
+        w = rec["workloads"][workload]
+        per_kernel = w["dram_bytes_per_param"]
+        return per_kernel[w["dominant"]] * units, sum(per_kernel.values()) * units
     except Exception:
-        return None
-    if rec.get("kernels_cuh_sha256_16") != kernel_source_hash() or workload not in rec.get("valid_for", []):
-        return None
-    return rec["dram_bytes_per_param"] * units
+        return None, None
 
 
 class ClockSampler:
@@ -290,15 +292,18 @@ def run_ours(args):
         upd_ms = ms_update / max(1, n_timed)
     achieved = update_bytes / (upd_ms * 1e-3) / 1e9
     kernel_name = "k_fused (sweep + decisions + update in one launch)" if fused else "k_apply (master update + cast)"
+    traffic_kernel, traffic_step = recorded_traffic(wl.name, wl.num_params)
     roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-                "traffic": recorded_traffic("k_fused" if fused else "k_apply", wl.name, wl.num_params),
+                "traffic": traffic_kernel,
                 "algorithmic_bytes_per_launch": update_bytes, "ms_per_launch": upd_ms,
                 "phases_ms_per_step": {"sweep": ms_sweep / max(1, n_timed), "decide_select": ms_decide / max(1, n_timed), "update": upd_ms},
                 "sweep_achieved_gbs": sweep_bytes / (ms_sweep / max(1, n_timed) * 1e-3) / 1e9,
                 "step": {"algorithmic_bytes": step_bytes_min, "achieved_gbs": step_bytes_min / (ms_step * 1e-3) / 1e9,
                          "frac_of_peak": step_bytes_min / (ms_step * 1e-3) / 1e9 / peak,
-                         "frac_of_8tbs_nominal": step_bytes_min / (ms_step * 1e-3) / 1e9 / 8000.0}}
+                         "frac_of_8tbs_nominal": step_bytes_min / (ms_step * 1e-3) / 1e9 / 8000.0,
+                         "dram_bytes_measured": traffic_step,
+                         "dram_gbs_measured": (traffic_step / (ms_step * 1e-3) / 1e9) if traffic_step else None}}
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
