@@ -20,7 +20,7 @@
 #define TA_SWEEP_ROWS_P1 8
 #endif
 #ifndef TA_SWEEP_ROWS_P1_BF16
-#define TA_SWEEP_ROWS_P1_BF16 16
+#define TA_SWEEP_ROWS_P1_BF16 8
 #endif
 #ifndef TA_SWEEP_ROWS_P2
 #define TA_SWEEP_ROWS_P2 4
