@@ -299,7 +299,8 @@ def run_ours(args):
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
                 "traffic": traffic_kernel,
                 "algorithmic_bytes_per_launch": update_bytes, "ms_per_launch": upd_ms,
-                "phases_ms_per_step": {"sweep": ms_sweep / max(1, n_timed), "decide_select": ms_decide / max(1, n_timed), "update": upd_ms},
+                "phases_ms_per_step": (None if fused else {"sweep": ms_sweep / max(1, n_timed), "decide_select": ms_decide / max(1, n_timed),
+                                                            "update": ms_update / max(1, n_timed)}),
                 "sweep_achieved_gbs": sweep_bytes / (ms_sweep / max(1, n_timed) * 1e-3) / 1e9,
                 "step": {"algorithmic_bytes": step_bytes_min, "achieved_gbs": step_bytes_min / (ms_step * 1e-3) / 1e9,
                          "frac_of_peak": step_bytes_min / (ms_step * 1e-3) / 1e9 / peak,
