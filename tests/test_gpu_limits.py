@@ -62,3 +62,36 @@ def test_thousands_of_tiny_layers(ppm, P):
     for t in (1, 2):
         g = torch.from_numpy((rng.standard_normal(n_total) * 1e-3).astype(np.float32)).cuda()
         run.step(t, g, oracle_hz(D, P, 5, t), 5)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_tables(seed):
+    # random tables, gaps, probe counts, mask fractions and gradient types: planner and kernels against the oracle
+    rng = np.random.default_rng(1000 + seed)
+    L = int(rng.integers(1, 40))
+    lengths = [int(rng.integers(1, 300)) if rng.random() < 0.7 else int(rng.integers(300, 30000)) for _ in range(L)]
+    table, off = [], int(rng.integers(0, 9))
+    for n in lengths:
+        off += int(rng.integers(0, 4)) * int(rng.random() < 0.5)
+        table.append((off, n))
+        off += n
+    n_total = (off + int(rng.integers(0, 9)) + 3) // 4 * 4
+    P = int(rng.choice([1, 2, 4, 8]))
+    ppm = 1000000 if rng.random() < 0.4 else int(rng.integers(1, 999999))
+    grad_dtype = "bf16" if rng.random() < 0.4 else "f32"
+    hp = dict(beta=float(rng.choice([0.0, 0.5, 0.9])), tau_low=3e-7, tau_high=3e-6, tau_curv=0.5, alpha=float(rng.choice([0.0, 1.0, 3.0])),
+              eta0=0.05, topk_ppm=ppm, num_probes=P, t_ctrl=int(rng.choice([1, 2])), grad_dtype=grad_dtype,
+              momentum=float(rng.choice([0.0, 0.0, 0.9])), weight_decay=float(rng.choice([0.0, 0.0, 1e-3])))
+    run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
+    D = np.exp(rng.uniform(np.log(1e-4), 0.5, n_total)).astype(np.float32)
+    if rng.random() < 0.5:
+        D = np.round(D * 8) / 8 + np.float32(0.125)          # few distinct values: many ties at the threshold
+    sigma = 10.0 ** rng.uniform(-4.5, -2.0, L)
+    for t in (1, 2, 3):
+        g = np.zeros(n_total, dtype=np.float32)
+        for (o, n), s in zip(table, sigma):
+            g[o:o + n] = rng.standard_normal(n) * s
+        g_dev = torch.from_numpy(g).cuda()
+        if grad_dtype == "bf16":
+            g_dev = g_dev.to(torch.bfloat16)
+        run.step(t, g_dev, oracle_hz(D, P, seed, t) if t != 2 else None, seed)
