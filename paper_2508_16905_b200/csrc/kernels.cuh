@@ -1325,15 +1325,14 @@ struct ResolveArgs {
 };
 
 // One block per layer: finishes the selection among the layer's candidates.
-__global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
+__device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32_t l)
 {
-    if (A.status->skipped) return;
     __shared__ uint32_t h[kHistBins];
     __shared__ uint32_t scan[kThreads];
     __shared__ uint32_t found[2];
     __shared__ double red[kWarps];
     __shared__ unsigned long long acc_u64[2];
-    const uint32_t l = blockIdx.x, tid = threadIdx.x;
+    const uint32_t tid = threadIdx.x;
     const uint64_t off = A.seg_off[l];
     SelectState s = A.sel[l];
     const uint32_t b1 = s.prefix;
@@ -1436,6 +1435,28 @@ __global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
         A.state[l].thr = __uint_as_float(thr);
         A.state[l].topk_mass = all > 0.0 ? (mass + cand_sum) / all : 1.0;
     }
+}
+
+__global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
+{
+    if (A.status->skipped) return;
+    resolve_layer(A, blockIdx.x);
+}
+
+// Top-k steps: the update needs nothing from the resolve step, so both run in ONE launch.  The first
+// n_layers blocks finish the selection of one layer each; the other blocks stride over the update batches.
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) k_apply_resolve(const ApplyArgs A, const ResolveArgs R, const uint32_t n_layers)
+{
+    if (A.status->skipped) return;
+    if (blockIdx.x < n_layers) {
+        resolve_layer(R, blockIdx.x);
+        return;
+    }
+    const LayerState *state = A.state;
+    // eta and code were fixed by k_decide; resolve blocks write other fields (threshold, mass) of the same records
+    auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
+    for (uint32_t batch = blockIdx.x - n_layers; batch < A.n_batches; batch += gridDim.x - n_layers) apply_batch<BF16>(A, batch, decision);
 }
 
 }  // namespace ta

@@ -60,7 +60,6 @@ struct ta_handle {
     cudaStream_t last_stream = nullptr;
     std::vector<cudaEvent_t> events;      // 4 per timed step: before sweep, after sweep, after decisions, after update
     uint32_t timed_cap = 0, timed_used = 0;
-    // top-k: the per-layer resolve kernel runs beside the update kernel on a stream of its own
     bool expire_next_wait = false;        // test aid: the next one-launch step waits for arrivals that never come
     bool fused_ok = false;                // small dense models: sweep + decisions + update in one cooperative launch
     int fused_grid[2][5] = {};            // resident grid of each k_fused variant: [bf16][index of P in 0,1,2,4,8]
@@ -69,8 +68,6 @@ struct ta_handle {
     cudaStream_t copy_back = nullptr;     // ta_step_host: device-to-host copies run beside the host-to-device ones
     std::vector<cudaEvent_t> chunk_done;
     cudaEvent_t decided = nullptr;
-    cudaStream_t side = nullptr;
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     DeviceBuffers d;
     char err[256] = "";
 };
@@ -268,9 +265,6 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     if (!h) return fail(nullptr, TA_ERR_NOMEM, "ta_create: out of host memory");
     auto bail = [&](int code) {
         snprintf(g_create_error, 256, "%s", h->err);
-        if (h->side) cudaStreamDestroy(h->side);
-        if (h->ev_fork) cudaEventDestroy(h->ev_fork);
-        if (h->ev_join) cudaEventDestroy(h->ev_join);
         free_all(h->d);
         delete h;
         return code;
@@ -398,9 +392,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         TA_TRY(dev_alloc(&d.cand_idx, n_total));
         TA_TRY(dev_alloc(&d.batch_seg, h->n_batches));
         TA_TRY(cudaMemset(d.cand_count, 0, (size_t)L * sizeof(uint32_t)));
-        TA_TRY(cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
-        TA_TRY(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
-        TA_TRY(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+
         TA_TRY(cudaMemcpy(d.batch_seg, batch_seg.data(), batch_seg.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
         TA_TRY(cudaMemset(d.hist, 0, (size_t)L * ta::kHistBins * sizeof(uint32_t)));
         TA_TRY(cudaMemset(d.sel, 0, (size_t)L * sizeof(ta::SelectState)));
@@ -445,12 +437,9 @@ int ta_destroy(ta_handle *h)
     cudaSetDevice(h->device);
     if (h->last_stream || h->stepped) cudaStreamSynchronize(h->last_stream);
     for (cudaEvent_t e : h->events) cudaEventDestroy(e);
-    if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
     if (h->copy_back) { cudaStreamSynchronize(h->copy_back); cudaStreamDestroy(h->copy_back); }
     for (cudaEvent_t e : h->chunk_done) cudaEventDestroy(e);
     if (h->decided) cudaEventDestroy(h->decided);
-    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
-    if (h->ev_join) cudaEventDestroy(h->ev_join);
     free_all(h->d);
     cudaSetDevice(prev);
     delete h;
@@ -589,17 +578,28 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
         ta::k_mask_compact<<<grid, ta::kThreads, 0, s>>>(ma);
         ta::ResolveArgs ra{d.item_lo, d.seg_off, d.seg_len, d.cand_count, d.cand_val, d.cand_idx, d.mask, d.p_mass,
                            d.scratch, d.sel, d.state, d.status};
-        // the update below needs nothing from the resolve step: run the two side by side
-        TA_CUDA(h, cudaEventRecord(h->ev_fork, s));
-        TA_CUDA(h, cudaStreamWaitEvent(h->side, h->ev_fork, 0));
-        ta::k_resolve<<<h->L, ta::kThreads, 0, h->side>>>(ra);
-        TA_CUDA(h, cudaEventRecord(h->ev_join, h->side));
+        // the update needs nothing from the resolve step: both run in one launch (k_apply_resolve) unless the
+        // caller applies the update itself
+        if (!defer_apply) {
+            if (timed) cudaEventRecord(ev[2], s);
+            ta::ApplyArgs aa{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status, d.mom, h->hp.momentum, h->hp.weight_decay};
+            const unsigned blocks = (unsigned)h->L + (unsigned)grid;
+            if (bf16) ta::k_apply_resolve<true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+            else ta::k_apply_resolve<false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+            h->launches += 2;
+            if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
+            TA_CUDA(h, cudaGetLastError());
+            h->stepped = true;
+            h->last_step = step;
+            h->last_stream = s;
+            return TA_OK;
+        }
+        ta::k_resolve<<<h->L, ta::kThreads, 0, s>>>(ra);
         h->launches += 2;
     }
 
     if (timed) cudaEventRecord(ev[2], s);
     if (!defer_apply) launch_apply(h, w, g, c, 0, h->n_items, s);
-    if (topk) TA_CUDA(h, cudaStreamWaitEvent(s, h->ev_join, 0));
     if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
 
     TA_CUDA(h, cudaGetLastError());
