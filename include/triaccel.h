@@ -232,8 +232,8 @@ int ta_timing_begin(ta_handle *h, uint32_t max_steps);
 int ta_timing_end(ta_handle *h, double *ms_sweep, double *ms_decide, double *ms_update, uint32_t *steps);
 
 /*
- * Failure detection.  Small dense models run as one cooperative launch whose blocks meet at two
- * grid-wide barriers.  Every such wait is bounded (a few hundred milliseconds): a block that gives up
+ * Failure detection.  Small dense models run as one cooperative launch whose blocks meet at a
+ * grid-wide barrier.  Every such wait is bounded (a few hundred milliseconds): a block that gives up
  * records it and returns, the step then changes neither weights, copies nor per-layer state, and the
  * next ta_stats / ta_precision_codes returns TA_ERR_CUDA once ("a bounded device-side wait ran out"),
  * after which the handle is usable again.  ta_test_expire_next_wait is a test aid: it makes the waits of

@@ -792,10 +792,11 @@ __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
 // ------------------------------------------------------------------ one launch for small models
 //
 // When the whole model is small, three launches cost more than the data movement.  k_fused runs the
-// sweep, the decisions and the update in ONE cooperative launch (every block resident), separated by
-// two grid-wide barriers.  The gradient (and the weights, prefetched during the sweep) is then still
-// in L2 when the update reads it.  Waits are bounded: a block that gives up sets status->device_error
-// and returns, so a lost block cannot hang the GPU.
+// sweep, the decisions and the update in ONE cooperative launch (every block resident).  The block
+// that finishes the last item of a layer decides that layer at once; one grid-wide barrier separates
+// "all layers decided" from the first write.  The gradient is then still in L2 when the update reads
+// it.  The wait is bounded: a block that gives up sets status->device_error and returns, so a lost
+// block cannot hang the GPU.
 
 // What the block that owns a layer publishes for all blocks between the two barriers.
 struct LayerVerdict {
@@ -816,6 +817,9 @@ struct FusedArgs {
     unsigned long long step;
     unsigned long long *barrier;    // arrivals, only ever incremented
     unsigned long long barrier_base;// arrivals before this launch
+    unsigned long long *layer_arrivals;   // [L] finished items per layer, only ever incremented
+    unsigned long long launch_index;      // one-launch steps before this one (since the counters were last cleared)
+    LayerState *staged;             // [L] new states, committed after the barrier unless the step is skipped
     uint32_t prefetch_w;
 };
 
@@ -843,6 +847,26 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsign
     return ok != 0u;
 }
 
+constexpr uint32_t kWarpCombineItems = 64;     // layers with at most this many items are combined by one warp
+
+// The layer's decisions from its combined sums: staged new state plus the verdict every block reads.
+__device__ __forceinline__ void publish_layer(const FusedArgs &A, uint32_t l, const LayerState &old, double n, double s1,
+                                              double s2, uint32_t amax, uint32_t amin, uint32_t bad)
+{
+    const double mu = s1 / n;
+    double var = s2 / n - mu * mu;
+    if (!(var > 0.0)) var = 0.0;
+    LayerScratch sc;
+    sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = bad; sc.amax = amax; sc.amin = amin;
+    uint32_t near;
+    const LayerState st = decide_layer(A.dp, old, sc, near);
+    A.staged[l] = st;
+    LayerVerdict v;
+    v.eta = st.eta;
+    v.code_bad = st.code | (bad ? 0x80000000u : 0u);
+    A.verdict[l] = v;
+}
+
 template <int P, bool BF16>
 __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
 {
@@ -851,65 +875,95 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
     uint32_t *sh_code = reinterpret_cast<uint32_t *>(dyn_smem) + A.L;    // [L]
     __shared__ double red[kWarps], red2[kWarps];
     __shared__ uint32_t red_u[2][kWarps];
+    __shared__ uint32_t done_layer[kWarps], n_done;
     const uint32_t tid = threadIdx.x;
     const unsigned long long G = gridDim.x;
 
-    // phase 1: sweep
-    if (blockIdx.x == 0 && tid == 0) A.status->near_stage = 0u;
-    for (uint32_t batch = blockIdx.x; batch < A.sweep.n_batches; batch += gridDim.x)
+    // phase 1: sweep.  After each batch the block reports, per layer, how many of the layer's items it has
+    // finished; the block whose report completes a layer combines that layer's item partials in a fixed
+    // order, takes the layer's decisions and publishes step size, code and non-finite flag, with the new
+    // state staged beside them.  When the barrier below opens, every layer has been decided.
+    for (uint32_t batch = blockIdx.x; batch < A.sweep.n_batches; batch += gridDim.x) {
+        if (tid == 0) n_done = 0u;
+        __syncthreads();
         sweep_batch<P, BF16, false>(A.sweep, batch, nullptr);
-    if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) return;
-
-    // phase 2: blocks share the layers.  The owner of a layer combines the layer's item partials in a fixed
-    // order, takes the layer's decisions, keeps the new state in registers and publishes step size, code and
-    // its non-finite flag for everybody.  At most kOwned layers per block.
-    constexpr int kOwned = 4;
-    LayerState mine[kOwned];
-    uint32_t n_owned = 0;
-    for (uint32_t l = blockIdx.x; l < A.L; l += gridDim.x) {
-        const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
-        // thread 0 fetches what it needs for the decision while the partials are on their way
-        LayerState old;
-        double n = 1.0;
-        if (tid == 0) { old = A.state[l]; n = (double)A.seg_len[l]; }
-        double s1 = 0.0, s2 = 0.0;
-        uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
-#pragma unroll 4
-        for (uint32_t i = lo + tid; i < hi; i += kThreads) {
-            s1 += __ldcg(A.sweep.p_s1 + i);
-            s2 += __ldcg(A.sweep.p_s2 + i);
-            bad |= __ldcg(A.sweep.p_bad + i);
-            if (P > 0) {
-                amax = max(amax, __ldcg(A.sweep.p_amax + i));
-                amin = min(amin, __ldcg(A.sweep.p_amin + i));
+        // lane 0 of each warp wrote its item's partials; it now reports the item to the item's layer
+        if ((tid & 31u) == 0u) {
+            const uint32_t it = batch * kWarps + (tid >> 5);
+            if (it < A.sweep.n_items) {
+                __threadfence();
+                const uint32_t seg = A.sweep.items[it].seg;
+                const unsigned long long want = (A.launch_index + 1ull) * (A.item_lo[seg + 1] - A.item_lo[seg]);
+                if (atomicAdd(A.layer_arrivals + seg, 1ull) + 1ull == want) done_layer[atomicAdd(&n_done, 1u)] = seg;
+                __threadfence();
             }
         }
-        s1 = warp_sum(s1);
-        s2 = warp_sum(s2);
-        amax = __reduce_max_sync(0xFFFFFFFFu, amax);
-        amin = __reduce_min_sync(0xFFFFFFFFu, amin);
         __syncthreads();
-        if ((tid & 31) == 0) { red[tid >> 5] = s1; red2[tid >> 5] = s2; red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
-        bad = (uint32_t)__syncthreads_or((int)bad);
-        if (tid == 0) {
-            s1 = 0.0; s2 = 0.0;
-            for (int w = 0; w < kWarps; ++w) { s1 += red[w]; s2 += red2[w]; }
-            for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
-            const double mu = s1 / n;
-            double var = s2 / n - mu * mu;
-            if (!(var > 0.0)) var = 0.0;
-            LayerScratch sc;
-            sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = bad; sc.amax = amax; sc.amin = amin;
-            uint32_t near;
-            const LayerState st = decide_layer(A.dp, old, sc, near);
-            if (n_owned < (uint32_t)kOwned) mine[n_owned] = st;
-            LayerVerdict v;
-            v.eta = st.eta;
-            v.code_bad = st.code | (bad ? 0x80000000u : 0u);
-            A.verdict[l] = v;
-            if (near) atomicAdd(&A.status->near_stage, 1u);
+        const uint32_t nd = n_done;
+        // layers with few items: one warp each, all at once (thousands of tiny tensors complete eight at a time)
+        {
+            const uint32_t wq = tid >> 5, lane = tid & 31u;
+            if (wq < nd) {
+                const uint32_t l = done_layer[wq];
+                const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
+                if (hi - lo <= kWarpCombineItems) {
+                    LayerState old;
+                    double n = 1.0;
+                    if (lane == 0) { old = A.state[l]; n = (double)A.seg_len[l]; }
+                    double s1 = 0.0, s2 = 0.0;
+                    uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
+                    for (uint32_t i = lo + lane; i < hi; i += 32) {
+                        s1 += __ldcg(A.sweep.p_s1 + i);
+                        s2 += __ldcg(A.sweep.p_s2 + i);
+                        bad |= __ldcg(A.sweep.p_bad + i);
+                        if (P > 0) {
+                            amax = max(amax, __ldcg(A.sweep.p_amax + i));
+                            amin = min(amin, __ldcg(A.sweep.p_amin + i));
+                        }
+                    }
+                    s1 = warp_sum(s1);
+                    s2 = warp_sum(s2);
+                    amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+                    amin = __reduce_min_sync(0xFFFFFFFFu, amin);
+                    bad = __reduce_or_sync(0xFFFFFFFFu, bad);
+                    if (lane == 0) publish_layer(A, l, old, n, s1, s2, amax, amin, bad);
+                }
+            }
         }
-        ++n_owned;
+        // layers with many items: the whole block, one after the other
+        for (uint32_t q = 0; q < nd; ++q) {
+            const uint32_t l = done_layer[q];
+            const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
+            if (hi - lo <= kWarpCombineItems) continue;
+            LayerState old;
+            double n = 1.0;
+            if (tid == 0) { old = A.state[l]; n = (double)A.seg_len[l]; }
+            double s1 = 0.0, s2 = 0.0;
+            uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
+#pragma unroll 4
+            for (uint32_t i = lo + tid; i < hi; i += kThreads) {
+                s1 += __ldcg(A.sweep.p_s1 + i);
+                s2 += __ldcg(A.sweep.p_s2 + i);
+                bad |= __ldcg(A.sweep.p_bad + i);
+                if (P > 0) {
+                    amax = max(amax, __ldcg(A.sweep.p_amax + i));
+                    amin = min(amin, __ldcg(A.sweep.p_amin + i));
+                }
+            }
+            s1 = warp_sum(s1);
+            s2 = warp_sum(s2);
+            amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+            amin = __reduce_min_sync(0xFFFFFFFFu, amin);
+            __syncthreads();
+            if ((tid & 31) == 0) { red[tid >> 5] = s1; red2[tid >> 5] = s2; red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
+            bad = (uint32_t)__syncthreads_or((int)bad);
+            if (tid == 0) {
+                s1 = 0.0; s2 = 0.0;
+                for (int w = 0; w < kWarps; ++w) { s1 += red[w]; s2 += red2[w]; }
+                for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
+                publish_layer(A, l, old, n, s1, s2, amax, amin, bad);
+            }
+        }
     }
     // DRAM is idle until the update starts: pull this block's weights into L2 while waiting
     if (A.prefetch_w) {
@@ -923,8 +977,7 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
             }
         }
     }
-
-    if (!grid_barrier(A.barrier, A.barrier_base + 2ull * G, A.status)) return;
+    if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) return;
 
     // every block reads all verdicts: is the step committed, and with which step sizes and codes
     uint32_t any_bad = 0u;
@@ -939,10 +992,7 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
     if (blockIdx.x == 0 && tid == 0) {
         A.status->step = A.step;
         A.status->skipped = any_bad ? 1u : 0u;
-        if (!any_bad) {
-            A.status->nonfinite = 0ull;
-            if (A.dp.control) A.status->near_count = A.status->near_stage;
-        }
+        if (!any_bad) A.status->nonfinite = 0ull;
     }
     if (any_bad) {
         // skipped step: nothing changes.  The exact count of non-finite values is summed by block 0.
@@ -954,12 +1004,19 @@ __global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
         }
         return;
     }
-    if (tid == 0) {
-        uint32_t j = 0;
-        for (uint32_t l = blockIdx.x; l < A.L && j < (uint32_t)kOwned; l += gridDim.x, ++j) A.state[l] = mine[j];
+    // the staged states become the layers' states (nobody reads them any more in this launch)
+    for (uint32_t l = blockIdx.x * kThreads + tid; l < A.L; l += gridDim.x * kThreads) {
+        const LayerState *src = A.staged + l;
+        LayerState st;
+        st.grad_mean = __ldcg(&src->grad_mean); st.grad_var = __ldcg(&src->grad_var); st.topk_mass = __ldcg(&src->topk_mass);
+        st.ema_mean = __ldcg(&src->ema_mean); st.ema_var = __ldcg(&src->ema_var);
+        st.lambda_max = __ldcg(&src->lambda_max); st.thr = __ldcg(&src->thr);
+        st.eta_scale = __ldcg(&src->eta_scale); st.eta = __ldcg(&src->eta);
+        st.code = __ldcg(&src->code); st.near = __ldcg(&src->near);
+        A.state[l] = st;
     }
 
-    // phase 3: update + cast
+    // phase 2: update + cast
     auto decision = [sh_eta, sh_code](uint32_t seg, float &eta, uint32_t &code) { eta = sh_eta[seg]; code = sh_code[seg]; };
     for (uint32_t batch = blockIdx.x; batch < A.apply.n_batches; batch += gridDim.x) apply_batch<BF16>(A.apply, batch, decision);
 }
