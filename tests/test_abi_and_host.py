@@ -161,3 +161,16 @@ print("rank", rank, "ok")
         pytest.skip("torchrun cannot take -c here")
     assert res.returncode == 0, res.stderr[-2000:]
     assert res.stdout.count("ok") == 2
+
+
+def test_reference_arm_of_the_benchmark_runs_on_cpu():
+    # `bench.py --impl reference` times the CPU checker; it must work without a GPU and print one JSON line
+    import json
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "mlp_tiny",
+                          "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=300,
+                         env=dict(os.environ, CUDA_VISIBLE_DEVICES=""))
+    assert res.returncode == 0, res.stderr[-1500:]
+    line = json.loads(res.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "params/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["config"]["workload"] == "mlp_tiny"
