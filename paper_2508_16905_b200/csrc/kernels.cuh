@@ -40,6 +40,16 @@
 #ifndef TA_APPLY_STREAM_W_STORE
 #define TA_APPLY_STREAM_W_STORE 0
 #endif
+// One-launch path: blocks per SM the compiler must leave room for, slots in flight in the sweep (P <= 1) and in the update.
+#ifndef TA_FUSED_MIN_BLOCKS
+#define TA_FUSED_MIN_BLOCKS 3
+#endif
+#ifndef TA_FUSED_SWEEP_SLOTS
+#define TA_FUSED_SWEEP_SLOTS 4
+#endif
+#ifndef TA_FUSED_UPDATE_SLOTS
+#define TA_FUSED_UPDATE_SLOTS 4
+#endif
 
 namespace ta {
 
@@ -138,6 +148,21 @@ __device__ __forceinline__ float4 ld_keep(const float *p)
     return __ldg(reinterpret_cast<const float4 *>(p));
 }
 
+// Loads that take no line of the L1 cache: for kernels that give most of the SM's memory to shared memory, where
+// the few lines left to L1 would otherwise bound the number of loads in flight.
+__device__ __forceinline__ float4 ld_no_l1(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ld_no_l1(const uint2 *p)
+{
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
 template <bool BF16> struct GradVec;
 template <> struct GradVec<false> {
     static __device__ __forceinline__ float4 load4(const void *g, uint64_t i, bool stream)
@@ -148,6 +173,10 @@ template <> struct GradVec<false> {
     static __device__ __forceinline__ float load1(const void *g, uint64_t i)
     {
         return __ldg(static_cast<const float *>(g) + i);
+    }
+    static __device__ __forceinline__ float4 load4_no_l1(const void *g, uint64_t i)
+    {
+        return ld_no_l1(static_cast<const float *>(g) + i);
     }
 };
 template <> struct GradVec<true> {
@@ -165,6 +194,16 @@ template <> struct GradVec<true> {
     static __device__ __forceinline__ float load1(const void *g, uint64_t i)
     {
         return __uint_as_float((uint32_t)__ldg(static_cast<const uint16_t *>(g) + i) << 16);
+    }
+    static __device__ __forceinline__ float4 load4_no_l1(const void *g, uint64_t i)
+    {
+        const uint2 v = ld_no_l1(reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(g) + i));
+        float4 r;
+        r.x = __uint_as_float(v.x << 16);
+        r.y = __uint_as_float(v.x & 0xFFFF0000u);
+        r.z = __uint_as_float(v.y << 16);
+        r.w = __uint_as_float(v.y & 0xFFFF0000u);
+        return r;
     }
 };
 
@@ -391,12 +430,14 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
         if (full_hi > full_lo) {
             uint64_t row = full_lo;
             RowData<P> rd[U];
-            // single rows up to the next multiple of U, so that an unrolled group never crosses a 32-row block
-            while (row < full_hi && (row & (U - 1))) {
+            // a short group up to the next multiple of U first, so that no group crosses a 32-row block (the probe
+            // bits of a lane are per block); needed only when probe bits are used
+            if (P > 1 && (row & (U - 1))) {
+                const int count = (int)min((uint64_t)U - (row & (U - 1)), full_hi - row);
                 refresh(row);
-                load_rows(row, rd, 1);
-                full_rows(row, rd, 1);
-                ++row;
+                load_rows(row, rd, count);
+                full_rows(row, rd, count);
+                row += count;
             }
             while (row + U <= full_hi) {
                 refresh(row);
@@ -404,11 +445,11 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                 full_rows(row, rd, U);
                 row += U;
             }
-            while (row < full_hi) {
+            if (row < full_hi) {
+                const int count = (int)(full_hi - row);
                 refresh(row);
-                load_rows(row, rd, 1);
-                full_rows(row, rd, 1);
-                ++row;
+                load_rows(row, rd, count);
+                full_rows(row, rd, count);
             }
         }
         if (tail_partial) partial_row(row_last);
@@ -792,38 +833,130 @@ __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
 // ------------------------------------------------------------------ one launch for small models
 //
 // When the whole model is small, three launches cost more than the data movement.  k_fused runs the
-// sweep, the decisions and the update in ONE cooperative launch (every block resident).  The block
-// that finishes the last item of a layer decides that layer at once; one grid-wide barrier separates
-// "all layers decided" from the first write.  The gradient is then still in L2 when the update reads
-// it.  The wait is bounded: a block that gives up sets status->device_error and returns, so a lost
-// block cannot hang the GPU.
+// sweep, the decisions and the update in ONE cooperative launch (every block resident) around one
+// grid-wide barrier.
+//
+// The plan gives every warp a list of "runs" (contiguous pieces of layers, the items of this path) of
+// equal total cost, cut on the global row grid.  A warp walks the rows of all its runs as one stream of
+// "slots" (a row plus the range of its elements that belong to the run; only the first and last row of
+// a layer are partial), several slots in flight, so a warp that owns a dozen tiny tensors waits for
+// memory as often as a warp that owns one long piece.  Before the barrier the warp accumulates the
+// statistics of its runs and parks as many of its gradient rows as fit in shared memory; its weights
+// travel to shared memory (cp.async, no registers held) while the grid waits at the barrier.  The block
+// folds the results of its runs into one partial per layer it touches.  After the barrier every block
+// combines, in a fixed order, the block partials of just the layers its own runs touch, takes their
+// decisions (every block arrives at identical values), and updates its slots from shared memory: nothing
+// is read from DRAM after the barrier except rows that did not fit.  The block holding a layer's first
+// run writes the layer's new state; old states were copied to shared memory before the barrier, so no
+// block can see a state of this step.  The wait is bounded: a block that gives up sets
+// status->device_error and returns, so a lost block cannot hang the GPU.
 
-// What the block that owns a layer publishes for all blocks between the two barriers.
-struct LayerVerdict {
-    float eta;           // step size of the layer if the step is committed
-    uint32_t code_bad;   // precision code in the low byte; bit 31: the layer saw a non-finite input
+// Statistics of one run, and of all runs of one layer inside one block.
+struct FusedPartial {
+    double s1, s2;               // sum and sum of squares of the gradient
+    uint32_t amax, amin;         // largest / smallest |S| as bit patterns
+    uint32_t bad, pad;           // non-finite inputs
+};
+
+// One slot: row `row` of the flat buffer, of which elements [lo, hi) (0..128 inside the row, packed as
+// lo | hi << 16) belong to run `run` (counted inside the warp) of layer `seg`.
+struct FusedSlot {
+    uint32_t row, lo_hi, run, seg;
+};
+
+// What the plan tells a warp and a block of the one-launch grid, and a block about each layer it touches.
+struct FusedWarpHead {
+    uint32_t run_lo, n_slots;        // first run of the warp, slots it walks
+    uint32_t pad0, pad1;
+};
+struct FusedBlockHead {
+    uint32_t run_lo, run_hi;         // runs of the block
+    uint32_t layer_lo, n_layers;     // layers they touch
+    uint32_t part_lo;                // first block partial (and first FusedBlockLayer) of the block
+    uint32_t pad0, pad1, pad2;
+};
+struct FusedBlockLayer {
+    double n;                        // length of the layer
+    uint32_t part_lo, part_hi;       // the layer's block partials
+    uint32_t own;                    // 1: this block holds the layer's first run and writes its state
+    uint32_t run_lo, run_hi;         // the layer's runs inside the block
+    uint32_t pad;
 };
 
 struct FusedArgs {
-    SweepArgs sweep;
-    ApplyArgs apply;
-    const uint32_t *item_lo;
-    const uint64_t *seg_len;
-    LayerVerdict *verdict;          // [L]
-    LayerState *state;              // [L]
+    const Item *runs;
+    uint32_t n_runs;
+    const void *g;
+    const float *hz;                    // [P][n_total] or unused when P == 0
+    uint64_t n_total;
+    uint64_t seed;
+    uint32_t step32;
+    float *w;
+    uint16_t *c;
+    const FusedWarpHead *warp_head;     // [warps]
+    const FusedBlockHead *block_head;   // [blocks]
+    const FusedBlockLayer *block_layer; // [n_part] one per (block, layer it touches), grouped by layer
+    const FusedSlot *slot_table;        // [warps][max_slots] the rows every warp walks
+    FusedPartial *part;                 // block partials, grouped by layer
+    uint32_t n_part;
+    LayerState *state;                  // [L]
     Status *status;
     DecideParams dp;
     uint32_t L;
+    uint32_t cap_w, cap_g;              // slots per warp whose weights / gradients stay in shared memory
+    uint32_t max_slots;                 // slots of the longest warp
+    uint32_t max_block_runs;            // runs of the block with most runs
+    uint32_t max_block_layers;          // layers of the block that touches most layers
+    uint32_t early_weights;             // 1: the weight copies start with the first loads of the sweep, 0: after the sweep
     unsigned long long step;
-    unsigned long long *barrier;    // arrivals, only ever incremented
-    unsigned long long barrier_base;// arrivals before this launch
-    unsigned long long *layer_arrivals;   // [L] finished items per layer, only ever incremented
-    unsigned long long launch_index;      // one-launch steps before this one (since the counters were last cleared)
-    LayerState *staged;             // [L] new states, committed after the barrier unless the step is skipped
-    uint32_t prefetch_w;
+    unsigned long long *barrier;        // [0] arrivals, only ever incremented; [1] last launch that saw non-finite input
+    unsigned long long barrier_base;    // arrivals before this launch
+    unsigned long long epoch;           // number of this launch (from 1)
 };
 
 constexpr uint32_t kBarrierSpinLimit = 1u << 20;     // with a 64 ns back-off: gives up after a few hundred milliseconds
+constexpr uint32_t kFusedMaxWarpRuns = 32;           // runs a warp may be given
+
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async16_once(void *smem, const void *gmem, uint64_t policy)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(s), "l"(gmem), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void *smem, const void *gmem)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// All groups of copies but the newest one have arrived.
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
+// Data that passes through L2 once is the first to leave it again; the plan, read by every launch, the last.
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ uint64_t l2_evict_last_policy()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ uint4 ld_plan(const void *p, uint64_t policy)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(policy));
+    return v;
+}
 
 // Grid-wide barrier on a monotonic arrival counter.  Returns false when the wait ran out.
 __device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsigned long long target, Status *status)
@@ -847,178 +980,320 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsign
     return ok != 0u;
 }
 
-constexpr uint32_t kWarpCombineItems = 64;     // layers with at most this many items are combined by one warp
-
-// The layer's decisions from its combined sums: staged new state plus the verdict every block reads.
-__device__ __forceinline__ void publish_layer(const FusedArgs &A, uint32_t l, const LayerState &old, double n, double s1,
-                                              double s2, uint32_t amax, uint32_t amin, uint32_t bad)
-{
-    const double mu = s1 / n;
-    double var = s2 / n - mu * mu;
-    if (!(var > 0.0)) var = 0.0;
-    LayerScratch sc;
-    sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = bad; sc.amax = amax; sc.amin = amin;
-    uint32_t near;
-    const LayerState st = decide_layer(A.dp, old, sc, near);
-    A.staged[l] = st;
-    LayerVerdict v;
-    v.eta = st.eta;
-    v.code_bad = st.code | (bad ? 0x80000000u : 0u);
-    A.verdict[l] = v;
-}
-
 template <int P, bool BF16>
-__global__ void __launch_bounds__(kThreads) k_fused(const FusedArgs A)
+__global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const FusedArgs A)
 {
-    extern __shared__ unsigned char dyn_smem[];
-    float *sh_eta = reinterpret_cast<float *>(dyn_smem);                 // [L]
-    uint32_t *sh_code = reinterpret_cast<uint32_t *>(dyn_smem) + A.L;    // [L]
-    __shared__ double red[kWarps], red2[kWarps];
-    __shared__ uint32_t red_u[2][kWarps];
-    __shared__ uint32_t done_layer[kWarps], n_done;
-    const uint32_t tid = threadIdx.x;
+    constexpr int PP = P > 0 ? P : 1;
+    constexpr int U = (P <= 1) ? TA_FUSED_SWEEP_SLOTS : (P == 2 ? 4 : 2);     // slots in flight per lane during the sweep
+    constexpr int UA = TA_FUSED_UPDATE_SLOTS;                                  // slots per group of the update
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const unsigned long long G = gridDim.x;
+    // dynamic shared memory: weight slots, gradient slots, slot descriptors (one slice per warp each), then the
+    // block's tables: what the plan says about its layers, results of its runs, old states and decisions
+    unsigned char *ptr = dyn_smem;
+    float4 *sh_w = reinterpret_cast<float4 *>(ptr) + (size_t)warp * A.cap_w * 32u;
+    ptr += (size_t)kWarps * A.cap_w * 512u;
+    float4 *sh_g = reinterpret_cast<float4 *>(ptr) + (size_t)warp * A.cap_g * 32u;
+    ptr += (size_t)kWarps * A.cap_g * 512u;
+    FusedSlot *sh_slot = reinterpret_cast<FusedSlot *>(ptr) + (size_t)warp * A.max_slots;
+    ptr += (size_t)kWarps * A.max_slots * sizeof(FusedSlot);
+    FusedBlockLayer *sh_bl = reinterpret_cast<FusedBlockLayer *>(ptr);
+    ptr += (size_t)A.max_block_layers * sizeof(FusedBlockLayer);
+    FusedPartial *sh_run = reinterpret_cast<FusedPartial *>(ptr);
+    ptr += (size_t)A.max_block_runs * sizeof(FusedPartial);
+    unsigned long long *sh_old = reinterpret_cast<unsigned long long *>(ptr);                          // LayerState each
+    ptr += (size_t)A.max_block_layers * sizeof(LayerState);
+    float *sh_eta = reinterpret_cast<float *>(ptr);
+    uint32_t *sh_code = reinterpret_cast<uint32_t *>(sh_eta + A.max_block_layers);
+    static_assert(sizeof(LayerState) % 8 == 0, "LayerState is copied as 64-bit words");
+    static_assert(sizeof(FusedSlot) == 16 && sizeof(FusedPartial) == 32, "shared-memory layout");
+    static_assert(sizeof(FusedWarpHead) == 16 && sizeof(FusedBlockHead) == 32 && sizeof(FusedBlockLayer) == 32, "plan records");
+    constexpr uint32_t kStateWords = sizeof(LayerState) / 8;
 
-    // phase 1: sweep.  After each batch the block reports, per layer, how many of the layer's items it has
-    // finished; the block whose report completes a layer combines that layer's item partials in a fixed
-    // order, takes the layer's decisions and publishes step size, code and non-finite flag, with the new
-    // state staged beside them.  When the barrier below opens, every layer has been decided.
-    for (uint32_t batch = blockIdx.x; batch < A.sweep.n_batches; batch += gridDim.x) {
-        if (tid == 0) n_done = 0u;
-        __syncthreads();
-        sweep_batch<P, BF16, false>(A.sweep, batch, nullptr);
-        // lane 0 of each warp wrote its item's partials; it now reports the item to the item's layer
-        if ((tid & 31u) == 0u) {
-            const uint32_t it = batch * kWarps + (tid >> 5);
-            if (it < A.sweep.n_items) {
-                __threadfence();
-                const uint32_t seg = A.sweep.items[it].seg;
-                const unsigned long long want = (A.launch_index + 1ull) * (A.item_lo[seg + 1] - A.item_lo[seg]);
-                if (atomicAdd(A.layer_arrivals + seg, 1ull) + 1ull == want) done_layer[atomicAdd(&n_done, 1u)] = seg;
-                __threadfence();
+    const uint64_t once = l2_evict_first_policy();       // the weights pass through L2 once on their way to shared memory
+    const uint64_t keep = l2_evict_last_policy();
+    // the plan of this warp and block: independent loads, one trip to L2
+    const uint32_t gw = blockIdx.x * kWarps + warp;
+    const uint4 wh = ld_plan(A.warp_head + gw, keep);
+    const uint4 bh0 = ld_plan(A.block_head + blockIdx.x, keep);
+    const uint4 bh1 = ld_plan(reinterpret_cast<const uint4 *>(A.block_head + blockIdx.x) + 1, keep);
+    for (uint32_t s = lane; s < A.max_slots; s += 32) {
+        const uint4 v = ld_plan(A.slot_table + (size_t)gw * A.max_slots + s, keep);
+        sh_slot[s] = FusedSlot{v.x, v.y, v.z, v.w};
+    }
+    const uint32_t run_lo = wh.x, n_slots = wh.y;
+    const uint32_t brun_lo = bh0.x, lf = bh0.z, nl = bh0.w, bpart_lo = bh1.x;
+    // the block's tables: its layers as the plan sees them, and the states the decisions start from, copied before
+    // anybody can have written a new one
+    for (uint32_t i = tid; i < nl * 2u; i += kThreads)
+        cp_async16(reinterpret_cast<uint4 *>(sh_bl) + i, reinterpret_cast<const uint4 *>(A.block_layer + bpart_lo) + i);
+    for (uint32_t i = tid; i < nl * kStateWords; i += kThreads)
+        cp_async8(sh_old + i, reinterpret_cast<const unsigned long long *>(A.state + lf) + i);
+    cp_async_commit();
+    __syncwarp();
+
+    // element range of this lane inside a slot: elements e of its vector with e_lo <= e < e_hi belong to the run
+    auto lane_range = [lane](const FusedSlot &sl, uint32_t &e_lo, uint32_t &e_hi) {
+        const uint32_t lo = sl.lo_hi & 0xFFFFu, hi = sl.lo_hi >> 16, l0 = lane * 4u;
+        e_lo = lo > l0 ? min(lo - l0, 4u) : 0u;
+        e_hi = hi < l0 + 4u ? (hi > l0 ? hi - l0 : 0u) : 4u;
+    };
+
+    // phase 1: statistics of this warp's runs (Sec. 3.1 moments; Sec. 3.2 probe sums)
+    {
+        SweepAcc<P, false> acc;
+        uint32_t X[PP][4];
+        uint64_t have_block = ~0ull;
+        uint32_t cur_run = 0u;
+        bool bad_seen = false;
+        auto flush = [&](uint32_t run) {
+            const double s1 = warp_sum(acc.s1), s2 = warp_sum(acc.s2);
+            const uint32_t amax = __reduce_max_sync(0xFFFFFFFFu, acc.amax);
+            const uint32_t amin = __reduce_min_sync(0xFFFFFFFFu, acc.amin);
+            const uint32_t gmax = __reduce_max_sync(0xFFFFFFFFu, acc.gmax);
+            uint32_t bad = 0u;
+            // a non-finite Hz value always makes its probe sum non-finite, so max|S| flags it
+            if (gmax >= kNonFiniteBits || (P > 0 && amax >= kNonFiniteBits)) {
+                // rare: count the non-finite inputs of this run exactly
+                const Item item = A.runs[run_lo + run];
+                for (uint64_t i = item.begin + lane; i < item.begin + item.len; i += 32) {
+                    if ((__float_as_uint(GradVec<BF16>::load1(A.g, i)) & 0x7FFFFFFFu) >= kNonFiniteBits) ++bad;
+                    for (int p = 0; p < P; ++p)
+                        if ((__float_as_uint(A.hz[(uint64_t)p * A.n_total + i]) & 0x7FFFFFFFu) >= kNonFiniteBits) ++bad;
+                }
+                bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+                bad_seen = bad_seen || bad != 0u;
             }
-        }
-        __syncthreads();
-        const uint32_t nd = n_done;
-        // layers with few items: one warp each, all at once (thousands of tiny tensors complete eight at a time)
-        {
-            const uint32_t wq = tid >> 5, lane = tid & 31u;
-            if (wq < nd) {
-                const uint32_t l = done_layer[wq];
-                const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
-                if (hi - lo <= kWarpCombineItems) {
-                    LayerState old;
-                    double n = 1.0;
-                    if (lane == 0) { old = A.state[l]; n = (double)A.seg_len[l]; }
-                    double s1 = 0.0, s2 = 0.0;
-                    uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
-                    for (uint32_t i = lo + lane; i < hi; i += 32) {
-                        s1 += __ldcg(A.sweep.p_s1 + i);
-                        s2 += __ldcg(A.sweep.p_s2 + i);
-                        bad |= __ldcg(A.sweep.p_bad + i);
-                        if (P > 0) {
-                            amax = max(amax, __ldcg(A.sweep.p_amax + i));
-                            amin = min(amin, __ldcg(A.sweep.p_amin + i));
+            if (lane == 0) sh_run[run_lo - brun_lo + run] = FusedPartial{s1, s2, amax, amin, bad, 0u};
+            acc = SweepAcc<P, false>();
+        };
+        auto start_weight_copies = [&]() {
+            const uint32_t n = min(n_slots, A.cap_w);
+            for (uint32_t s = 0; s < n; ++s) {
+                const FusedSlot sl = sh_slot[s];
+                uint32_t e_lo, e_hi;
+                lane_range(sl, e_lo, e_hi);
+                if (e_hi > e_lo) cp_async16_once(sh_w + s * 32u + lane, A.w + (uint64_t)sl.row * 128ull + lane * 4u, once);
+            }
+            cp_async_commit();
+        };
+        for (uint32_t s0 = 0; s0 < n_slots; s0 += U) {
+            RowData<P> rd[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (s0 + u < n_slots) {
+                    const FusedSlot sl = sh_slot[s0 + u];
+                    uint32_t e_lo, e_hi;
+                    lane_range(sl, e_lo, e_hi);
+                    if (e_hi > e_lo) {
+                        const uint64_t i0 = (uint64_t)sl.row * 128ull + lane * 4u;
+                        // a gradient row that will wait in shared memory needs no place in L1 or L2; one that the
+                        // update reads again stays in L2 (a load without an L1 line is also among the first to
+                        // leave L2); probe products are read once
+                        rd[u].g = s0 + u < A.cap_g ? GradVec<BF16>::load4_no_l1(A.g, i0) : GradVec<BF16>::load4(A.g, i0, false);
+#pragma unroll
+                        for (int p = 0; p < PP; ++p)
+                            if (P > 0) rd[u].hz[p] = ld_stream(A.hz + (uint64_t)p * A.n_total + i0);
+                    }
+                }
+            }
+            if (s0 == 0 && A.early_weights) start_weight_copies();
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (s0 + u < n_slots) {
+                    const FusedSlot sl = sh_slot[s0 + u];
+                    if (sl.run != cur_run) { flush(cur_run); cur_run = sl.run; }
+                    uint32_t e_lo, e_hi;
+                    lane_range(sl, e_lo, e_hi);
+                    uint32_t sel[PP];
+                    const uint32_t k = sl.row & 31u;
+                    if (P > 1) {
+                        const uint64_t blk = sl.row >> 5;
+                        if (blk != have_block) {
+#pragma unroll
+                            for (int p = 0; p < PP; ++p) probe_bits(blk, lane, A.seed, A.step32, (uint32_t)p, X[p]);
+                            have_block = blk;
                         }
                     }
-                    s1 = warp_sum(s1);
-                    s2 = warp_sum(s2);
-                    amax = __reduce_max_sync(0xFFFFFFFFu, amax);
-                    amin = __reduce_min_sync(0xFFFFFFFFu, amin);
-                    bad = __reduce_or_sync(0xFFFFFFFFu, bad);
-                    if (lane == 0) publish_layer(A, l, old, n, s1, s2, amax, amin, bad);
+#pragma unroll
+                    for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
+                    const float gv[4] = {rd[u].g.x, rd[u].g.y, rd[u].g.z, rd[u].g.w};
+#pragma unroll
+                    for (uint32_t e = 0; e < 4; ++e) {
+                        if (e >= e_lo && e < e_hi) {
+                            float hv[PP];
+#pragma unroll
+                            for (int p = 0; p < PP; ++p) {
+                                const float4 h = rd[u].hz[p];
+                                hv[p] = e == 0 ? h.x : (e == 1 ? h.y : (e == 2 ? h.z : h.w));
+                            }
+                            acc.element(gv[e], hv, sel, (k & 7u) * 4u + e);
+                        }
+                    }
+                    if (s0 + u < A.cap_g && e_hi > e_lo) sh_g[(s0 + u) * 32u + lane] = rd[u].g;
                 }
             }
         }
-        // layers with many items: the whole block, one after the other
-        for (uint32_t q = 0; q < nd; ++q) {
-            const uint32_t l = done_layer[q];
-            const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
-            if (hi - lo <= kWarpCombineItems) continue;
-            LayerState old;
-            double n = 1.0;
-            if (tid == 0) { old = A.state[l]; n = (double)A.seg_len[l]; }
-            double s1 = 0.0, s2 = 0.0;
-            uint32_t amax = 0u, amin = 0xFFFFFFFFu, bad = 0u;
-#pragma unroll 4
-            for (uint32_t i = lo + tid; i < hi; i += kThreads) {
-                s1 += __ldcg(A.sweep.p_s1 + i);
-                s2 += __ldcg(A.sweep.p_s2 + i);
-                bad |= __ldcg(A.sweep.p_bad + i);
-                if (P > 0) {
-                    amax = max(amax, __ldcg(A.sweep.p_amax + i));
-                    amin = min(amin, __ldcg(A.sweep.p_amin + i));
-                }
-            }
-            s1 = warp_sum(s1);
-            s2 = warp_sum(s2);
-            amax = __reduce_max_sync(0xFFFFFFFFu, amax);
-            amin = __reduce_min_sync(0xFFFFFFFFu, amin);
-            __syncthreads();
-            if ((tid & 31) == 0) { red[tid >> 5] = s1; red2[tid >> 5] = s2; red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
-            bad = (uint32_t)__syncthreads_or((int)bad);
-            if (tid == 0) {
-                s1 = 0.0; s2 = 0.0;
-                for (int w = 0; w < kWarps; ++w) { s1 += red[w]; s2 += red2[w]; }
-                for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
-                publish_layer(A, l, old, n, s1, s2, amax, amin, bad);
-            }
-        }
+        if (n_slots) flush(cur_run);
+        // the weights arrive while the grid waits at the barrier and takes the decisions
+        if (!A.early_weights || n_slots == 0) start_weight_copies();
+        if (bad_seen && lane == 0) atomicMax(A.barrier + 1, A.epoch);
     }
-    // DRAM is idle until the update starts: pull this block's weights into L2 while waiting
-    if (A.prefetch_w) {
-        for (uint32_t batch = blockIdx.x; batch < A.sweep.n_batches; batch += gridDim.x) {
-            const uint32_t it = batch * kWarps + (tid >> 5);
-            if (it < A.sweep.n_items) {
-                const Item item = A.sweep.items[it];
-                const char *base = reinterpret_cast<const char *>(A.apply.w + item.begin);
-                for (uint32_t off = (tid & 31u) * 128u; off < item.len * 4u; off += 32u * 128u)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
-            }
+    // the block's runs folded into one partial per layer it touches, in run order
+    cp_async_wait_but_one();        // the block's tables have arrived (the weight copies may still be under way)
+    __syncthreads();
+    if (tid < nl) {
+        const uint32_t lo = sh_bl[tid].run_lo, hi = sh_bl[tid].run_hi;
+        FusedPartial t{0.0, 0.0, 0u, 0xFFFFFFFFu, 0u, 0u};
+        for (uint32_t r = lo; r < hi; ++r) {
+            const FusedPartial x = sh_run[r - brun_lo];
+            t.s1 += x.s1; t.s2 += x.s2;
+            t.amax = max(t.amax, x.amax); t.amin = min(t.amin, x.amin);
+            t.bad += x.bad;
         }
+        A.part[bpart_lo + tid] = t;
     }
-    if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) return;
 
-    // every block reads all verdicts: is the step committed, and with which step sizes and codes
-    uint32_t any_bad = 0u;
-    for (uint32_t l = tid; l < A.L; l += kThreads) {
-        const float eta = __ldcg(&A.verdict[l].eta);
-        const uint32_t cb = __ldcg(&A.verdict[l].code_bad);
-        sh_eta[l] = eta;
-        sh_code[l] = cb & 0xFFu;
-        any_bad |= cb >> 31;
+    if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) {
+        cp_async_wait_all();
+        return;
     }
-    any_bad = (uint32_t)__syncthreads_or((int)any_bad);      // also orders the shared-memory table before its use
+
+    const bool skip = __ldcg(A.barrier + 1) == A.epoch;
     if (blockIdx.x == 0 && tid == 0) {
         A.status->step = A.step;
-        A.status->skipped = any_bad ? 1u : 0u;
-        if (!any_bad) A.status->nonfinite = 0ull;
+        A.status->skipped = skip ? 1u : 0u;
+        if (!skip) A.status->nonfinite = 0ull;
     }
-    if (any_bad) {
+    if (skip) {
         // skipped step: nothing changes.  The exact count of non-finite values is summed by block 0.
         if (blockIdx.x == 0) {
+            __shared__ double red[kWarps];
             double total = 0.0;
-            for (uint32_t i = tid; i < A.sweep.n_items; i += kThreads) total += (double)__ldcg(A.sweep.p_bad + i);
+            for (uint32_t i = tid; i < A.n_part; i += kThreads) total += (double)__ldcg(&A.part[i].bad);
             total = block_sum(total, red);
             if (tid == 0) A.status->nonfinite = (unsigned long long)total;
         }
+        cp_async_wait_all();
         return;
     }
-    // the staged states become the layers' states (nobody reads them any more in this launch)
-    for (uint32_t l = blockIdx.x * kThreads + tid; l < A.L; l += gridDim.x * kThreads) {
-        const LayerState *src = A.staged + l;
-        LayerState st;
-        st.grad_mean = __ldcg(&src->grad_mean); st.grad_var = __ldcg(&src->grad_var); st.topk_mass = __ldcg(&src->topk_mass);
-        st.ema_mean = __ldcg(&src->ema_mean); st.ema_var = __ldcg(&src->ema_var);
-        st.lambda_max = __ldcg(&src->lambda_max); st.thr = __ldcg(&src->thr);
-        st.eta_scale = __ldcg(&src->eta_scale); st.eta = __ldcg(&src->eta);
-        st.code = __ldcg(&src->code); st.near = __ldcg(&src->near);
-        A.state[l] = st;
-    }
 
-    // phase 2: update + cast
-    auto decision = [sh_eta, sh_code](uint32_t seg, float &eta, uint32_t &code) { eta = sh_eta[seg]; code = sh_code[seg]; };
-    for (uint32_t batch = blockIdx.x; batch < A.apply.n_batches; batch += gridDim.x) apply_batch<BF16>(A.apply, batch, decision);
+    // decisions of the layers this block touches, from the block partials of each (Sec. 3.1 - 3.4)
+    auto decide = [&](uint32_t q, double s1, double s2, uint32_t amax, uint32_t amin) {
+        LayerState old;
+        unsigned long long *dst = reinterpret_cast<unsigned long long *>(&old);
+#pragma unroll
+        for (uint32_t i = 0; i < kStateWords; ++i) dst[i] = sh_old[q * kStateWords + i];
+        const double n = sh_bl[q].n;
+        const double mu = s1 / n;
+        double var = s2 / n - mu * mu;
+        if (!(var > 0.0)) var = 0.0;
+        LayerScratch sc;
+        sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = 0ull; sc.amax = amax; sc.amin = amin;
+        uint32_t near;
+        const LayerState st = decide_layer(A.dp, old, sc, near);
+        sh_eta[q] = st.eta;
+        sh_code[q] = st.code;
+        if (sh_bl[q].own) A.state[lf + q] = st;
+    };
+    constexpr uint32_t kThreadCombine = 4;       // layers with at most this many block partials: one thread each
+    for (uint32_t q = tid; q < nl; q += kThreads) {
+        const uint32_t lo = sh_bl[q].part_lo, hi = sh_bl[q].part_hi;
+        if (hi - lo > kThreadCombine) continue;
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+        for (uint32_t i = lo; i < hi; ++i) {
+            s1 += __ldcg(&A.part[i].s1);
+            s2 += __ldcg(&A.part[i].s2);
+            amax = max(amax, __ldcg(&A.part[i].amax));
+            amin = min(amin, __ldcg(&A.part[i].amin));
+        }
+        decide(q, s1, s2, amax, amin);
+    }
+    for (uint32_t q = warp; q < nl; q += kWarps) {      // layers spread over many blocks: one warp each
+        const uint32_t lo = sh_bl[q].part_lo, hi = sh_bl[q].part_hi;
+        if (hi - lo <= kThreadCombine) continue;
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+        for (uint32_t i = lo + lane; i < hi; i += 32) {
+            s1 += __ldcg(&A.part[i].s1);
+            s2 += __ldcg(&A.part[i].s2);
+            amax = max(amax, __ldcg(&A.part[i].amax));
+            amin = min(amin, __ldcg(&A.part[i].amin));
+        }
+        s1 = warp_sum(s1);
+        s2 = warp_sum(s2);
+        amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+        amin = __reduce_min_sync(0xFFFFFFFFu, amin);
+        if (lane == 0) decide(q, s1, s2, amax, amin);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+
+    // phase 2: update + cast of this warp's slots (Sec. 3.2 step, Sec. 2 master copy and cast)
+    for (uint32_t s0 = 0; s0 < n_slots; s0 += UA) {
+        float4 wv[UA], gv[UA];
+#pragma unroll
+        for (int u = 0; u < UA; ++u) {
+            const uint32_t s = s0 + u;
+            if (s < n_slots) {
+                const FusedSlot sl = sh_slot[s];
+                uint32_t e_lo, e_hi;
+                lane_range(sl, e_lo, e_hi);
+                if (e_hi > e_lo) {
+                    const uint64_t i0 = (uint64_t)sl.row * 128ull + lane * 4u;
+                    wv[u] = s < A.cap_w ? sh_w[s * 32u + lane] : ld_stream(A.w + i0);
+                    gv[u] = s < A.cap_g ? sh_g[s * 32u + lane] : GradVec<BF16>::load4(A.g, i0, true);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UA; ++u) {
+            const uint32_t s = s0 + u;
+            if (s < n_slots) {
+                const FusedSlot sl = sh_slot[s];
+                uint32_t e_lo, e_hi;
+                lane_range(sl, e_lo, e_hi);
+                if (e_hi > e_lo) {
+                    const uint64_t i0 = (uint64_t)sl.row * 128ull + lane * 4u;
+                    const float neg_eta = -sh_eta[sl.seg - lf];
+                    const uint32_t code = sh_code[sl.seg - lf];
+                    float4 x = wv[u];
+                    x.x = fmaf(neg_eta, gv[u].x, x.x);
+                    x.y = fmaf(neg_eta, gv[u].y, x.y);
+                    x.z = fmaf(neg_eta, gv[u].z, x.z);
+                    x.w = fmaf(neg_eta, gv[u].w, x.w);
+                    if (e_lo == 0u && e_hi == 4u) {
+                        *reinterpret_cast<float4 *>(A.w + i0) = x;
+                        if (code == 0u) {
+                            const __half2 a = __floats2half2_rn(x.x, x.y), b = __floats2half2_rn(x.z, x.w);
+                            uint2 o;
+                            o.x = *reinterpret_cast<const uint32_t *>(&a);
+                            o.y = *reinterpret_cast<const uint32_t *>(&b);
+                            __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
+                        } else if (code == 1u) {
+                            const __nv_bfloat162 a = __floats2bfloat162_rn(x.x, x.y), b = __floats2bfloat162_rn(x.z, x.w);
+                            uint2 o;
+                            o.x = *reinterpret_cast<const uint32_t *>(&a);
+                            o.y = *reinterpret_cast<const uint32_t *>(&b);
+                            __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
+                        }
+                    } else {
+                        // a vector on the edge of the layer: only the elements of this run are written
+                        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                        for (uint32_t e = 0; e < 4; ++e) {
+                            if (e >= e_lo && e < e_hi) {
+                                A.w[i0 + e] = xs[e];
+                                if (code < 2u) A.c[i0 + e] = cast16(xs[e], code);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------ power iteration support (Sec. 3.2)

@@ -22,10 +22,12 @@ struct DeviceBuffers {
     ta::LayerState *state = nullptr;
     ta::LayerScratch *scratch = nullptr;
     ta::Status *status = nullptr;
-    ta::LayerVerdict *verdict = nullptr;          // fused launch: per-layer step size, code, non-finite flag
-    unsigned long long *barrier = nullptr;        // fused launch: grid-barrier arrivals
-    unsigned long long *layer_arrivals = nullptr; // fused launch: finished items per layer
-    ta::LayerState *staged = nullptr;             // fused launch: new per-layer states until the step is committed
+    unsigned long long *barrier = nullptr;        // fused launch: [0] grid-barrier arrivals, [1] last launch with non-finite input
+    ta::FusedWarpHead *warp_head = nullptr;       // fused launch: the plan's records per warp, per block, per (block, layer)
+    ta::FusedBlockHead *block_head = nullptr;
+    ta::FusedBlockLayer *block_layer = nullptr;
+    ta::FusedSlot *slot_table = nullptr;
+    ta::FusedPartial *part = nullptr;             // fused launch: block partials, grouped by layer
     double *p_s1 = nullptr, *p_s2 = nullptr, *p_sa = nullptr, *p_mass = nullptr;
     uint32_t *p_amax = nullptr, *p_amin = nullptr, *p_bad = nullptr;
     float *abs_s = nullptr;
@@ -64,7 +66,10 @@ struct ta_handle {
     uint32_t timed_cap = 0, timed_used = 0;
     bool expire_next_wait = false;        // test aid: the next one-launch step waits for arrivals that never come
     bool fused_ok = false;                // small dense models: sweep + decisions + update in one cooperative launch
-    int fused_grid[2][5] = {};            // resident grid of each k_fused variant: [bf16][index of P in 0,1,2,4,8]
+    int fused_grid = 0;                   // blocks of the one-launch grid (all resident)
+    uint32_t fused_cap_w = 0, fused_cap_g = 0;                           // shared-memory slots per warp: weights, gradients
+    uint32_t fused_block_layers = 0, fused_block_runs = 0, fused_slots = 0, fused_parts = 0;   // table sizes of the plan
+    size_t fused_smem = 0;
     unsigned long long barrier_base = 0;  // barrier arrivals of all fused launches so far
     unsigned long long fused_launches = 0;// fused launches since the arrival counters were last cleared
     std::vector<ta::Item> items_host;     // the plan, kept for the pipelined host path
@@ -101,7 +106,7 @@ template <typename T> cudaError_t dev_alloc(T **p, size_t count)
 
 void free_all(DeviceBuffers &d)
 {
-    void *ptrs[] = {d.layer_arrivals, d.staged, d.mom, d.pw_part, d.pw_coef, d.pw_norm, d.verdict, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
+    void *ptrs[] = {d.warp_head, d.block_head, d.block_layer, d.slot_table, d.part, d.mom, d.pw_part, d.pw_coef, d.pw_norm, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
                     d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
     for (void *p : ptrs)
@@ -177,8 +182,6 @@ void launch_apply(ta_handle *h, float *w, const void *g, uint16_t *c, uint32_t i
     ++h->launches;
 }
 
-int p_index(int P) { return P == 0 ? 0 : P == 1 ? 1 : P == 2 ? 2 : P == 4 ? 3 : 4; }
-
 template <int P, bool BF16> const void *fused_fn() { return reinterpret_cast<const void *>(&ta::k_fused<P, BF16>); }
 
 const void *fused_kernel(int P, bool bf16)
@@ -191,6 +194,120 @@ const void *fused_kernel(int P, bool bf16)
     case 8: return bf16 ? fused_fn<8, true>() : fused_fn<8, false>();
     default: return nullptr;
     }
+}
+
+constexpr int kFusedSmemMax = 226 * 1024;         // dynamic shared memory a block may ask for (227 KB opt-in limit minus the static part)
+constexpr uint64_t kRunOverhead = 256;            // cost of starting a run, in elements: reductions and partial rows
+constexpr uint64_t kMinWarpCost = 512;            // a warp is given at least this much work
+
+// The plan of the one-launch path: every layer is cut into runs so that each of n_warps warps gets a list of
+// consecutive runs of equal total cost (elements plus a constant per run).  Cuts lie on the global grid of
+// 128-element rows, so only the first and the last row of a layer can be partial.
+struct RunPlan {
+    std::vector<ta::Item> runs;
+    std::vector<uint32_t> item_lo, warp_lo;           // first run of every layer / warp
+    std::vector<uint32_t> part_lo, block_part_lo;     // block partials: first of every layer, first of every block
+    std::vector<ta::FusedWarpHead> warp_head;
+    std::vector<ta::FusedBlockHead> block_head;
+    std::vector<ta::FusedBlockLayer> block_layer;
+    std::vector<ta::FusedSlot> slot_table;            // [n_warps][max_slots]
+    uint32_t n_warps = 0, n_part = 0;
+    uint32_t max_slots = 0, max_warp_runs = 0, max_block_runs = 0, max_block_layers = 0;
+};
+
+RunPlan plan_runs(const ta_segment *table, uint32_t L, uint64_t max_warps)
+{
+    RunPlan pl;
+    uint64_t cost = 0;
+    for (uint32_t l = 0; l < L; ++l) cost += table[l].length + kRunOverhead;
+    uint64_t n_warps = std::min<uint64_t>(max_warps, (cost + kMinWarpCost - 1) / kMinWarpCost);
+    n_warps = std::max<uint64_t>(ta::kWarps, (n_warps + ta::kWarps - 1) / ta::kWarps * ta::kWarps);
+    const double target = (double)cost / (double)n_warps;
+    pl.n_warps = (uint32_t)n_warps;
+    pl.item_lo.resize(L + 1);
+    std::vector<uint32_t> run_warp;
+    uint64_t cum = 0, warp = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        pl.item_lo[l] = (uint32_t)pl.runs.size();
+        const uint64_t b = table[l].offset, e = b + table[l].length;
+        cum += kRunOverhead;
+        for (uint64_t p = b; p < e;) {
+            const double room = target * (double)(warp + 1) - (double)cum;
+            uint64_t q = e;
+            if (warp + 1 < n_warps && room < (double)(e - p)) {
+                q = (p + (uint64_t)std::max(room, 0.0) + 64) / 128 * 128;        // nearest row boundary
+                if (q <= p) q = (p / 128 + 1) * 128;
+                if (q > e) q = e;
+            }
+            pl.runs.push_back(ta::Item{p, (uint32_t)(q - p), l});
+            run_warp.push_back((uint32_t)warp);
+            cum += q - p;
+            p = q;
+            while (warp + 1 < n_warps && (double)cum >= target * (double)(warp + 1) - 64.0) ++warp;      // this warp is full
+        }
+    }
+    pl.item_lo[L] = (uint32_t)pl.runs.size();
+    pl.warp_lo.assign(n_warps + 1, (uint32_t)pl.runs.size());
+    for (size_t r = pl.runs.size(); r-- > 0;) pl.warp_lo[run_warp[r]] = (uint32_t)r;
+    for (size_t wq = n_warps; wq-- > 0;) pl.warp_lo[wq] = std::min(pl.warp_lo[wq], pl.warp_lo[wq + 1]);   // warps without runs
+    for (uint64_t wq = 0; wq < n_warps; ++wq) {
+        uint64_t slots = 0;       // rows the warp visits, partial ones included
+        for (uint32_t r = pl.warp_lo[wq]; r < pl.warp_lo[wq + 1]; ++r)
+            slots += (pl.runs[r].begin + pl.runs[r].len - 1) / 128 - pl.runs[r].begin / 128 + 1;
+        pl.max_slots = std::max<uint32_t>(pl.max_slots, (uint32_t)slots);
+        pl.max_warp_runs = std::max(pl.max_warp_runs, pl.warp_lo[wq + 1] - pl.warp_lo[wq]);
+    }
+    // every block writes one partial per layer it touches; in (block, layer) order these are grouped by layer
+    const uint64_t n_blocks = n_warps / ta::kWarps;
+    pl.block_part_lo.resize(n_blocks);
+    std::vector<uint32_t> per_layer(L, 0);
+    for (uint64_t blk = 0; blk < n_blocks; ++blk) {
+        const uint32_t lo = pl.warp_lo[blk * ta::kWarps], hi = pl.warp_lo[(blk + 1) * ta::kWarps];
+        pl.block_part_lo[blk] = pl.n_part;
+        if (hi <= lo) continue;
+        const uint32_t lf = pl.runs[lo].seg, ll = pl.runs[hi - 1].seg;
+        pl.max_block_layers = std::max(pl.max_block_layers, ll - lf + 1);
+        pl.max_block_runs = std::max(pl.max_block_runs, hi - lo);
+        for (uint32_t l = lf; l <= ll; ++l) ++per_layer[l];
+        pl.n_part += ll - lf + 1;
+    }
+    pl.part_lo.resize(L + 1);
+    pl.part_lo[0] = 0;
+    for (uint32_t l = 0; l < L; ++l) pl.part_lo[l + 1] = pl.part_lo[l] + per_layer[l];
+    // the records the kernel reads: per warp its slots, per block its runs and layers
+    pl.warp_head.assign(n_warps, ta::FusedWarpHead{0, 0, 0, 0});
+    pl.slot_table.assign((size_t)n_warps * pl.max_slots, ta::FusedSlot{0, 0, 0, 0});
+    for (uint64_t wq = 0; wq < n_warps; ++wq) {
+        uint32_t n = 0;
+        for (uint32_t r = pl.warp_lo[wq]; r < pl.warp_lo[wq + 1]; ++r) {
+            const uint64_t b = pl.runs[r].begin, e = b + pl.runs[r].len;
+            for (uint64_t row = b / 128; row <= (e - 1) / 128; ++row) {
+                const uint64_t r0 = row * 128;
+                const uint32_t lo = b > r0 ? (uint32_t)(b - r0) : 0u, hi = e < r0 + 128 ? (uint32_t)(e - r0) : 128u;
+                pl.slot_table[wq * pl.max_slots + n++] = ta::FusedSlot{(uint32_t)row, lo | (hi << 16), r - pl.warp_lo[wq], pl.runs[r].seg};
+            }
+        }
+        pl.warp_head[wq] = ta::FusedWarpHead{pl.warp_lo[wq], n, 0, 0};
+    }
+    pl.block_head.resize(n_blocks);
+    pl.block_layer.resize(pl.n_part);
+    for (uint64_t blk = 0; blk < n_blocks; ++blk) {
+        const uint32_t lo = pl.warp_lo[blk * ta::kWarps], hi = pl.warp_lo[(blk + 1) * ta::kWarps];
+        const uint32_t lf = hi > lo ? pl.runs[lo].seg : 0u, nl = hi > lo ? pl.runs[hi - 1].seg - lf + 1 : 0u;
+        pl.block_head[blk] = ta::FusedBlockHead{lo, hi, lf, nl, pl.block_part_lo[blk], 0, 0, 0};
+        for (uint32_t q = 0; q < nl; ++q) {
+            const uint32_t l = lf + q;
+            ta::FusedBlockLayer bl{};
+            bl.n = (double)table[l].length;
+            bl.part_lo = pl.part_lo[l];
+            bl.part_hi = pl.part_lo[l + 1];
+            bl.own = pl.item_lo[l] >= lo ? 1u : 0u;
+            bl.run_lo = std::max(pl.item_lo[l], lo);
+            bl.run_hi = std::min(pl.item_lo[l + 1], hi);
+            pl.block_layer[pl.block_part_lo[blk] + q] = bl;
+        }
+    }
+    return pl;
 }
 
 uint64_t fused_max_params()
@@ -208,8 +325,7 @@ int check_device_error(ta_handle *h)
     if (!s.device_error) return TA_OK;
     s.device_error = 0u;
     TA_CUDA(h, cudaMemcpy(h->d.status, &s, sizeof(s), cudaMemcpyHostToDevice));
-    if (h->d.barrier) TA_CUDA(h, cudaMemset(h->d.barrier, 0, sizeof(unsigned long long)));
-    if (h->d.layer_arrivals) TA_CUDA(h, cudaMemset(h->d.layer_arrivals, 0, h->L * sizeof(unsigned long long)));
+    if (h->d.barrier) TA_CUDA(h, cudaMemset(h->d.barrier, 0, 2 * sizeof(unsigned long long)));
     h->barrier_base = 0;
     h->fused_launches = 0;
     return fail(h, TA_ERR_CUDA, "a bounded device-side wait ran out during the last step; its results are incomplete");
@@ -299,48 +415,70 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     h->mask_words = h->topk ? (n_total + 31) / 32 : 0;
 
     // one-launch path for small dense models: needs a cooperative launch with every block resident
-    long long fused_blocks = 0;
+    int fused_per_sm = 0;
     {
         int coop = 0;
         TA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device));
-        const size_t smem = (size_t)L * 8;
-        if (coop && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f && n_params <= fused_max_params() && smem <= 32 * 1024) {
+        if (coop && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f && n_params <= fused_max_params()) {
             const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
             h->fused_ok = true;
-            fused_blocks = 1ll << 40;
+            fused_per_sm = 1 << 20;
             for (int P : {0, (int)hp->num_probes}) {
                 int per_sm = 0;
-                TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(P, bf16), ta::kThreads, smem));
-                if (const char *env = getenv("TRIACCEL_FUSED_CTAS_PER_SM")) per_sm = std::min(per_sm, std::max(1, atoi(env)));
-                h->fused_grid[bf16][p_index(P)] = per_sm * h->sm_count;
-                fused_blocks = std::min<long long>(fused_blocks, (long long)per_sm * h->sm_count);
-                if (per_sm < 1) h->fused_ok = false;
+                TA_TRY(cudaFuncSetAttribute(fused_kernel(P, bf16), cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemMax));
+                TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(P, bf16), ta::kThreads, 0));
+                fused_per_sm = std::min(fused_per_sm, per_sm);
             }
+            if (const char *env = getenv("TRIACCEL_FUSED_CTAS_PER_SM")) fused_per_sm = std::min(fused_per_sm, std::max(1, atoi(env)));
+            if (fused_per_sm < 1) h->fused_ok = false;
         }
     }
 
     // plan: items cut on a global grid of item_elems elements, clipped to each layer
     h->item_elems = choose_item_elems(n_params, h->sm_count);
-    if (h->fused_ok && !getenv("TRIACCEL_ITEM_ELEMS")) {
-        // one item per warp of the resident grid if the model is small enough: every phase is a single round
-        for (uint32_t cand = 512; cand <= 16384; cand += 512) {
-            unsigned long long count = 0;
-            for (uint32_t l = 0; l < L; ++l)
-                count += (table[l].offset + table[l].length - 1) / cand - table[l].offset / cand + 1;
-            if (count <= (unsigned long long)fused_blocks * ta::kWarps) { h->item_elems = cand; break; }
-        }
-    }
     std::vector<ta::Item> items;
     std::vector<uint32_t> item_lo(L + 1);
+    RunPlan run_plan;
     std::vector<uint64_t> seg_off(L), seg_len(L);
     h->seg_k.resize(L);
     for (uint32_t l = 0; l < L; ++l) {
-        item_lo[l] = (uint32_t)items.size();
-        const uint64_t b = table[l].offset, e = b + table[l].length;
-        seg_off[l] = b;
+        seg_off[l] = table[l].offset;
         seg_len[l] = table[l].length;
         uint64_t k = (table[l].length * (uint64_t)hp->topk_ppm + 999999ull) / 1000000ull;
         h->seg_k[l] = k < 1 ? 1 : k;
+    }
+    if (h->fused_ok) {
+        // one-launch path: the items are the runs of a plan that gives every resident warp the same amount of work;
+        // what is left of the SM's shared memory, after the per-block tables, holds weight rows first, then gradient rows
+        RunPlan pl = plan_runs(table, L, (uint64_t)h->sm_count * fused_per_sm * ta::kWarps);
+        const size_t tables = (size_t)pl.max_block_layers * (sizeof(ta::LayerState) + sizeof(ta::FusedBlockLayer) + 8) +
+                              (size_t)pl.max_block_runs * sizeof(ta::FusedPartial) + (size_t)ta::kWarps * pl.max_slots * sizeof(ta::FusedSlot);
+        const long long per_block = std::min<long long>(kFusedSmemMax, (228ll * 1024) / fused_per_sm - 1024) - 512 /* static */ - (long long)tables;
+        const long long rows_fit = per_block / (ta::kWarps * 512);
+        if (rows_fit < 0 || tables > 64 * 1024 || pl.max_warp_runs > ta::kFusedMaxWarpRuns || n_total >= (1ull << 38)) {
+            h->fused_ok = false;
+        } else {
+            // weights first, then gradients; a model whose weights do not all fit gains nothing from a part of
+            // them (its update is bound by the write-back of what it writes): it keeps nothing in shared memory
+            h->fused_cap_w = (uint32_t)std::min<long long>(pl.max_slots, rows_fit);
+            h->fused_cap_g = (uint32_t)std::min<long long>(pl.max_slots, rows_fit - h->fused_cap_w);
+            if (h->fused_cap_w < pl.max_slots) h->fused_cap_w = h->fused_cap_g = 0;
+            if (const char *env = getenv("TRIACCEL_FUSED_CAP_W")) h->fused_cap_w = std::min<uint32_t>(h->fused_cap_w, (uint32_t)atoi(env));
+            if (const char *env = getenv("TRIACCEL_FUSED_CAP_G")) h->fused_cap_g = std::min<uint32_t>(h->fused_cap_g, (uint32_t)atoi(env));
+            h->fused_block_layers = pl.max_block_layers;
+            h->fused_block_runs = pl.max_block_runs;
+            h->fused_slots = pl.max_slots;
+            h->fused_parts = pl.n_part;
+            h->fused_smem = (size_t)ta::kWarps * 512 * (h->fused_cap_w + h->fused_cap_g) + tables;
+            h->fused_grid = (int)(pl.n_warps / ta::kWarps);
+            items = pl.runs;
+            item_lo = pl.item_lo;
+            run_plan = std::move(pl);
+        }
+    }
+    for (uint32_t l = 0; l < L && !h->fused_ok; ++l) {
+        item_lo[l] = (uint32_t)items.size();
+        const uint64_t b = table[l].offset, e = b + table[l].length;
         // top-k: a layer of at least one full batch starts on a batch boundary, so that its batches hold one
         // layer only and can count their histogram in shared memory (padding items are empty)
         const uint64_t layer_items = (e - 1) / h->item_elems - b / h->item_elems + 1;
@@ -354,7 +492,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         }
         if (items.size() > 0x7FFFFFFFull) { snprintf(h->err, 256, "ta_create: too many work items"); return bail(TA_ERR_ARG); }
     }
-    item_lo[L] = (uint32_t)items.size();
+    if (!h->fused_ok) item_lo[L] = (uint32_t)items.size();
     h->items_host = items;
     h->n_items = (uint32_t)items.size();
     h->n_batches = (h->n_items + ta::kWarps - 1) / ta::kWarps;
@@ -423,12 +561,27 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         TA_TRY(cudaMemset(d.mom, 0, n_total * sizeof(float)));
     }
     if (h->fused_ok) {
-        TA_TRY(dev_alloc(&d.verdict, L));
-        TA_TRY(dev_alloc(&d.barrier, 1));
-        TA_TRY(cudaMemset(d.barrier, 0, sizeof(unsigned long long)));
-        TA_TRY(dev_alloc(&d.layer_arrivals, L));
-        TA_TRY(cudaMemset(d.layer_arrivals, 0, L * sizeof(unsigned long long)));
-        TA_TRY(dev_alloc(&d.staged, L));
+        TA_TRY(dev_alloc(&d.barrier, 2));
+        TA_TRY(cudaMemset(d.barrier, 0, 2 * sizeof(unsigned long long)));
+        TA_TRY(dev_alloc(&d.warp_head, run_plan.warp_head.size()));
+        TA_TRY(cudaMemcpy(d.warp_head, run_plan.warp_head.data(), run_plan.warp_head.size() * sizeof(ta::FusedWarpHead), cudaMemcpyHostToDevice));
+        TA_TRY(dev_alloc(&d.block_head, run_plan.block_head.size()));
+        TA_TRY(cudaMemcpy(d.block_head, run_plan.block_head.data(), run_plan.block_head.size() * sizeof(ta::FusedBlockHead), cudaMemcpyHostToDevice));
+        TA_TRY(dev_alloc(&d.block_layer, run_plan.block_layer.size()));
+        TA_TRY(cudaMemcpy(d.block_layer, run_plan.block_layer.data(), run_plan.block_layer.size() * sizeof(ta::FusedBlockLayer), cudaMemcpyHostToDevice));
+        TA_TRY(dev_alloc(&d.slot_table, run_plan.slot_table.size()));
+        TA_TRY(cudaMemcpy(d.slot_table, run_plan.slot_table.data(), run_plan.slot_table.size() * sizeof(ta::FusedSlot), cudaMemcpyHostToDevice));
+        TA_TRY(dev_alloc(&d.part, h->fused_parts));
+        // the occupancy the plan counted on must hold with the shared memory it asks for
+        const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
+        for (int P : {0, (int)hp->num_probes}) {
+            int per_sm = 0;
+            TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(P, bf16), ta::kThreads, h->fused_smem));
+            if ((long long)per_sm * h->sm_count < h->fused_grid) {
+                snprintf(h->err, 256, "ta_create: the one-launch grid of %d blocks is not resident (%d per SM)", h->fused_grid, per_sm);
+                return bail(TA_ERR_CUDA);
+            }
+        }
     }
     TA_TRY(cudaDeviceSynchronize());
 #undef TA_TRY
@@ -531,24 +684,25 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
 
     if (h->fused_ok) {
         ta::FusedArgs fa{};
-        fa.sweep.items = d.items; fa.sweep.n_items = h->n_items; fa.sweep.n_batches = h->n_batches;
-        fa.sweep.g = g; fa.sweep.hz = Hz; fa.sweep.n_total = h->n_total; fa.sweep.seed = probe_seed; fa.sweep.step = (uint32_t)step;
-        fa.sweep.p_s1 = d.p_s1; fa.sweep.p_s2 = d.p_s2; fa.sweep.p_sa = d.p_sa;
-        fa.sweep.p_amax = d.p_amax; fa.sweep.p_amin = d.p_amin; fa.sweep.p_bad = d.p_bad;
-        fa.apply = ta::ApplyArgs{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status, nullptr, 0.f, 0.f};
-        fa.item_lo = d.item_lo; fa.seg_len = d.seg_len; fa.verdict = d.verdict;
+        fa.runs = d.items; fa.n_runs = h->n_items;
+        fa.g = g; fa.hz = Hz; fa.n_total = h->n_total; fa.seed = probe_seed; fa.step32 = (uint32_t)step;
+        fa.w = w; fa.c = c;
+        fa.warp_head = d.warp_head; fa.block_head = d.block_head; fa.block_layer = d.block_layer; fa.slot_table = d.slot_table;
+        fa.part = d.part; fa.n_part = h->fused_parts;
         fa.state = d.state; fa.status = d.status;
         fa.dp.hp = hyper_of(h->hp); fa.dp.eta0 = h->hp.eta0; fa.dp.has_hz = Hz ? 1u : 0u;
         fa.dp.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; fa.dp.topk = 0u;
-        fa.L = h->L; fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base;
-        fa.layer_arrivals = d.layer_arrivals; fa.launch_index = h->fused_launches; fa.staged = d.staged;
+        fa.L = h->L; fa.cap_w = h->fused_cap_w; fa.cap_g = h->fused_cap_g;
+        fa.max_slots = h->fused_slots; fa.max_block_runs = h->fused_block_runs; fa.max_block_layers = h->fused_block_layers;
+        fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base;
+        fa.epoch = h->fused_launches + 1;
+        // the weight copies start after the sweep (measured faster than starting them with its first loads)
+        static const bool early_w = getenv("TRIACCEL_FUSED_EARLY_W") ? atoi(getenv("TRIACCEL_FUSED_EARLY_W")) != 0 : false;
+        fa.early_weights = early_w ? 1u : 0u;
         if (h->expire_next_wait) { fa.barrier_base += 1ull << 40; h->expire_next_wait = false; }
-        // weight prefetch into L2 before the barrier: measured neutral on the EfficientNet-B0 mix and a loss on ResNet-18
-        static const bool prefetch = getenv("TRIACCEL_FUSED_PREFETCH") ? atoi(getenv("TRIACCEL_FUSED_PREFETCH")) != 0 : false;
-        fa.prefetch_w = prefetch ? 1u : 0u;
-        const int grid = (int)std::min<long long>(h->fused_grid[bf16][p_index(P)], h->n_batches);
+        const int grid = h->fused_grid;
         void *args[] = {&fa};
-        TA_CUDA(h, cudaLaunchCooperativeKernel(fused_kernel(P, bf16), dim3(grid), dim3(ta::kThreads), args, (size_t)h->L * 8, s));
+        TA_CUDA(h, cudaLaunchCooperativeKernel(fused_kernel(P, bf16), dim3(grid), dim3(ta::kThreads), args, h->fused_smem, s));
         h->barrier_base += (unsigned long long)grid;
         ++h->fused_launches;
         ++h->launches;
