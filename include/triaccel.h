@@ -242,6 +242,27 @@ int ta_timing_end(ta_handle *h, double *ms_sweep, double *ms_decide, double *ms_
  */
 int ta_test_expire_next_wait(ta_handle *h);
 
+/*
+ * The work plan of the one-launch path, for inspection (host only, no GPU needed).  Small dense models
+ * run the whole pass of Sec. 3.1 - 3.2 in one launch; its plan cuts every layer into "runs" (contiguous
+ * pieces, cut on the grid of 128-element rows of the flat buffer, so that only the first and last row
+ * of a layer can be partial) and gives each of at most `warps` warps a list of consecutive runs of
+ * about equal cost (elements plus a constant per run), which is what keeps a table of thousands of
+ * tiny tensors beside a few large ones from starving warps.  Writes the runs in buffer order to
+ * out[0 .. *n_runs) (at most cap; TA_ERR_ARG if there are more), the number of warps that got work to
+ * *warps_used and the largest number of rows one warp walks to *max_rows.  ta_create builds the same
+ * plan with warps = resident warps of the device.  Table rules as for ta_create.
+ */
+typedef struct ta_run {
+    uint64_t begin;      /* first element */
+    uint32_t length;     /* elements, all inside one layer */
+    uint32_t layer;
+    uint32_t warp;       /* the warp of the grid that handles the run */
+    uint32_t reserved;
+} ta_run;
+int ta_plan_one_launch(const ta_segment *table, uint32_t L, uint32_t warps, ta_run *out, uint32_t cap,
+                       uint32_t *n_runs, uint32_t *warps_used, uint32_t *max_rows);
+
 /* Static description of the last error of this handle ("" if none).  h may be NULL: then the
  * last ta_create failure of the calling thread. */
 const char *ta_last_error(const ta_handle *h);

@@ -21,11 +21,16 @@ EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "t
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
            "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
            "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait",
-           "ta_power_iterate", "ta_set_curvature"]
+           "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch"]
 
 
 class ta_segment(C.Structure):
     _fields_ = [("offset", C.c_uint64), ("length", C.c_uint64)]
+
+
+class ta_run(C.Structure):
+    _fields_ = [("begin", C.c_uint64), ("length", C.c_uint32), ("layer", C.c_uint32), ("warp", C.c_uint32),
+                ("reserved", C.c_uint32)]
 
 
 class ta_hparams(C.Structure):
@@ -96,6 +101,8 @@ def lib():
     L.ta_test_expire_next_wait.argtypes = [vp]
     L.ta_power_iterate.argtypes = [vp, vp, vp, vp, vp, u32, vp, vp, vp, vp]
     L.ta_set_curvature.argtypes = [vp, vp]
+    L.ta_plan_one_launch.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_run), u32, C.POINTER(u32), C.POINTER(u32),
+                                     C.POINTER(u32)]
     L.ta_static_last_error.argtypes = []
     L.ta_static_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -268,6 +275,19 @@ def ta_set_curvature(h, lambda_max):
     if a.size != h.L:
         raise ValueError("one value per layer")
     _check(lib().ta_set_curvature(h.ptr, a.ctypes.data_as(C.c_void_p)), h.ptr)
+
+
+def ta_plan_one_launch(table, warps):
+    """table: sequence of (offset, length). Returns (runs as a list of (begin, length, layer, warp), warps_used, max_rows)."""
+    L = len(table)
+    segs = (ta_segment * max(L, 1))(*[ta_segment(int(o), int(n)) for o, n in table])
+    n, used, rows = C.c_uint32(), C.c_uint32(), C.c_uint32()
+    cap = L + int(warps) + 8
+    out = (ta_run * cap)()
+    rc = lib().ta_plan_one_launch(segs, L, int(warps), out, cap, C.byref(n), C.byref(used), C.byref(rows))
+    if rc != TA_OK:
+        raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
+    return [(r.begin, r.length, r.layer, r.warp) for r in out[:n.value]], used.value, rows.value
 
 
 def ta_test_expire_next_wait(h):

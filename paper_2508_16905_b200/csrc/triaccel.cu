@@ -455,7 +455,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
                               (size_t)pl.max_block_runs * sizeof(ta::FusedPartial) + (size_t)ta::kWarps * pl.max_slots * sizeof(ta::FusedSlot);
         const long long per_block = std::min<long long>(kFusedSmemMax, (228ll * 1024) / fused_per_sm - 1024) - 512 /* static */ - (long long)tables;
         const long long rows_fit = per_block / (ta::kWarps * 512);
-        if (rows_fit < 0 || tables > 64 * 1024 || pl.max_warp_runs > ta::kFusedMaxWarpRuns || n_total >= (1ull << 38)) {
+        if (rows_fit < 0 || tables > 64 * 1024 || n_total >= (1ull << 38)) {
             h->fused_ok = false;
         } else {
             // weights first, then gradients; a model whose weights do not all fit gains nothing from a part of
@@ -626,6 +626,32 @@ int ta_test_expire_next_wait(ta_handle *h)
     if (!h) return TA_ERR_ARG;
     if (!h->fused_ok) return fail(h, TA_ERR_STATE, "ta_test_expire_next_wait: this handle does not use the one-launch path");
     h->expire_next_wait = true;
+    return TA_OK;
+}
+
+int ta_plan_one_launch(const ta_segment *table, uint32_t L, uint32_t warps, ta_run *out, uint32_t cap,
+                       uint32_t *n_runs, uint32_t *warps_used, uint32_t *max_rows)
+{
+    if (!table || L == 0 || warps == 0 || !n_runs) return fail(nullptr, TA_ERR_ARG, "ta_plan_one_launch: table, L, warps and n_runs are required");
+    uint64_t end = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        if (table[l].length == 0 || table[l].length > 0xFFFFFFFEull)
+            return fail(nullptr, TA_ERR_ARG, "ta_plan_one_launch: segment length out of range");
+        if (table[l].offset < end) return fail(nullptr, TA_ERR_ARG, "ta_plan_one_launch: segments must be ascending and non-overlapping");
+        end = table[l].offset + table[l].length;
+    }
+    const RunPlan pl = plan_runs(table, L, warps);
+    *n_runs = (uint32_t)pl.runs.size();
+    if (warps_used) {
+        uint32_t used = 0;
+        for (uint32_t wq = 0; wq < pl.n_warps; ++wq) used += pl.warp_lo[wq + 1] > pl.warp_lo[wq] ? 1u : 0u;
+        *warps_used = used;
+    }
+    if (max_rows) *max_rows = pl.max_slots;
+    if (pl.runs.size() > cap || (!out && cap)) return fail(nullptr, TA_ERR_ARG, "ta_plan_one_launch: out is too small for the plan");
+    for (uint32_t wq = 0; wq < pl.n_warps; ++wq)
+        for (uint32_t r = pl.warp_lo[wq]; r < pl.warp_lo[wq + 1]; ++r)
+            out[r] = ta_run{pl.runs[r].begin, pl.runs[r].len, pl.runs[r].seg, wq, 0u};
     return TA_OK;
 }
 

@@ -174,3 +174,74 @@ def test_reference_arm_of_the_benchmark_runs_on_cpu():
     assert line["impl"] == "reference" and line["unit"] == "params/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["config"]["workload"] == "mlp_tiny"
+
+
+# ---------------------------------------------------------------- plan of the one-launch path (host logic)
+
+def _check_plan(table, warps):
+    from paper_2508_16905_b200 import binding as B
+    runs, used, max_rows = B.ta_plan_one_launch(table, warps)
+    # the runs tile every layer exactly, in buffer order, and interior cuts lie on the 128-element row grid
+    by_layer = {}
+    for begin, length, layer, warp in runs:
+        assert length > 0
+        by_layer.setdefault(layer, []).append((begin, length))
+    assert sorted(by_layer) == list(range(len(table)))
+    for l, (off, n) in enumerate(table):
+        pos = off
+        for begin, length in by_layer[l]:
+            assert begin == pos
+            pos += length
+            if pos != off + n:
+                assert pos % 128 == 0
+        assert pos == off + n
+    # warps get consecutive runs; no warp index beyond the request; about equal cost
+    warps_seen = [w for *_, w in runs]
+    assert warps_seen == sorted(warps_seen) and warps_seen[-1] < max(8, -(-warps // 8) * 8)
+    assert used == len(set(warps_seen))
+    cost, rows = {}, {}
+    for begin, length, layer, w in runs:
+        cost[w] = cost.get(w, 0) + length
+        rows[w] = rows.get(w, 0) + (begin + length - 1) // 128 - begin // 128 + 1
+    n_layers_cost = 256 * len(table)
+    total = sum(n for _, n in table) + n_layers_cost
+    n_warps = max(8, -(-min(warps, -(-total // 512)) // 8) * 8)
+    target = total / n_warps
+    assert max(cost.values()) <= target + 128 + 64, (max(cost.values()), target)
+    assert max_rows == max(rows.values())
+    return runs, used, max_rows
+
+
+def test_one_launch_plan_on_the_benchmark_tables():
+    from paper_2508_16905_b200 import workloads as W
+    for name in ("mlp_tiny", "resnet18_cifar", "efficientnet_b0_cifar"):
+        wl = W.get(name)
+        for warps in (8, 148 * 8, 148 * 24, 148 * 32):
+            _check_plan(wl.table, warps)
+    # the EfficientNet-B0 mix on a full B200 grid: every warp has work and walks a dozen rows at most
+    wl = W.get("efficientnet_b0_cifar")
+    runs, used, max_rows = _check_plan(wl.table, 148 * 24)
+    assert used == 148 * 24 and max_rows <= 14
+
+
+def test_one_launch_plan_on_random_tables():
+    import numpy as np
+    rng = np.random.default_rng(7)
+    for trial in range(60):
+        L = int(rng.integers(1, 400))
+        lens = np.where(rng.random(L) < 0.6, rng.integers(1, 300, L), rng.integers(300, 200000, L))
+        gaps = rng.integers(0, 50, L) * (rng.random(L) < 0.5)
+        table, pos = [], 0
+        for n, gap in zip(lens, gaps):
+            pos += int(gap)
+            table.append((pos, int(n)))
+            pos += int(n)
+        _check_plan(table, int(rng.choice([8, 64, 1184, 3552, 4736])))
+
+
+def test_one_launch_plan_rejects_bad_tables():
+    from paper_2508_16905_b200 import binding as B
+    with pytest.raises(B.TriAccelError):
+        B.ta_plan_one_launch([(0, 10), (5, 10)], 64)          # overlapping
+    with pytest.raises(B.TriAccelError):
+        B.ta_plan_one_launch([(0, 0)], 64)                    # empty segment
