@@ -430,14 +430,12 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
         if (full_hi > full_lo) {
             uint64_t row = full_lo;
             RowData<P> rd[U];
-            // a short group up to the next multiple of U first, so that no group crosses a 32-row block (the probe
-            // bits of a lane are per block); needed only when probe bits are used
-            if (P > 1 && (row & (U - 1))) {
-                const int count = (int)min((uint64_t)U - (row & (U - 1)), full_hi - row);
+            // single rows up to the next multiple of U, so that an unrolled group never crosses a 32-row block
+            while (row < full_hi && (row & (U - 1))) {
                 refresh(row);
-                load_rows(row, rd, count);
-                full_rows(row, rd, count);
-                row += count;
+                load_rows(row, rd, 1);
+                full_rows(row, rd, 1);
+                ++row;
             }
             while (row + U <= full_hi) {
                 refresh(row);
@@ -445,11 +443,11 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                 full_rows(row, rd, U);
                 row += U;
             }
-            if (row < full_hi) {
-                const int count = (int)(full_hi - row);
+            while (row < full_hi) {
                 refresh(row);
-                load_rows(row, rd, count);
-                full_rows(row, rd, count);
+                load_rows(row, rd, 1);
+                full_rows(row, rd, 1);
+                ++row;
             }
         }
         if (tail_partial) partial_row(row_last);
@@ -915,7 +913,6 @@ struct FusedArgs {
 };
 
 constexpr uint32_t kBarrierSpinLimit = 1u << 20;     // with a 64 ns back-off: gives up after a few hundred milliseconds
-constexpr uint32_t kFusedMaxWarpRuns = 32;           // runs a warp may be given
 
 __device__ __forceinline__ void cp_async16(void *smem, const void *gmem)
 {
@@ -1160,24 +1157,9 @@ __global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const F
         return;
     }
 
+    // did any warp of the grid see a non-finite input?  The answer is needed only when results are committed, so
+    // the decisions below are taken while it is on its way; those of a skipped step are thrown away
     const bool skip = __ldcg(A.barrier + 1) == A.epoch;
-    if (blockIdx.x == 0 && tid == 0) {
-        A.status->step = A.step;
-        A.status->skipped = skip ? 1u : 0u;
-        if (!skip) A.status->nonfinite = 0ull;
-    }
-    if (skip) {
-        // skipped step: nothing changes.  The exact count of non-finite values is summed by block 0.
-        if (blockIdx.x == 0) {
-            __shared__ double red[kWarps];
-            double total = 0.0;
-            for (uint32_t i = tid; i < A.n_part; i += kThreads) total += (double)__ldcg(&A.part[i].bad);
-            total = block_sum(total, red);
-            if (tid == 0) A.status->nonfinite = (unsigned long long)total;
-        }
-        cp_async_wait_all();
-        return;
-    }
 
     // decisions of the layers this block touches, from the block partials of each (Sec. 3.1 - 3.4)
     auto decide = [&](uint32_t q, double s1, double s2, uint32_t amax, uint32_t amin) {
@@ -1195,7 +1177,7 @@ __global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const F
         const LayerState st = decide_layer(A.dp, old, sc, near);
         sh_eta[q] = st.eta;
         sh_code[q] = st.code;
-        if (sh_bl[q].own) A.state[lf + q] = st;
+        if (sh_bl[q].own && !skip) A.state[lf + q] = st;
     };
     constexpr uint32_t kThreadCombine = 4;       // layers with at most this many block partials: one thread each
     for (uint32_t q = tid; q < nl; q += kThreads) {
@@ -1229,6 +1211,22 @@ __global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const F
         if (lane == 0) decide(q, s1, s2, amax, amin);
     }
     cp_async_wait_all();
+    if (blockIdx.x == 0 && tid == 0) {
+        A.status->step = A.step;
+        A.status->skipped = skip ? 1u : 0u;
+        if (!skip) A.status->nonfinite = 0ull;
+    }
+    if (skip) {
+        // skipped step: nothing changes.  The exact count of non-finite values is summed by block 0.
+        if (blockIdx.x == 0) {
+            __shared__ double red[kWarps];
+            double total = 0.0;
+            for (uint32_t i = tid; i < A.n_part; i += kThreads) total += (double)__ldcg(&A.part[i].bad);
+            total = block_sum(total, red);
+            if (tid == 0) A.status->nonfinite = (unsigned long long)total;
+        }
+        return;
+    }
     __syncthreads();
 
     // phase 2: update + cast of this warp's slots (Sec. 3.2 step, Sec. 2 master copy and cast)
