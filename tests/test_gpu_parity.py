@@ -208,6 +208,43 @@ def test_non_finite_input_skips_the_whole_step():
     assert ta.ta_stats(run.h)[1].skipped == 0
 
 
+def test_non_finite_input_skips_the_whole_step_one_launch():
+    """Dense model on the one-launch path: bad values in a one-element layer, on the partial last row of a layer
+    and in two layers at once; the exact count is reported, nothing changes, and the next clean step matches."""
+    table, n_total = ragged_table([1, 33, 5000, 2, 300, 70000, 129, 7])
+    rng = np.random.default_rng(3)
+    hp = dict(num_probes=1, tau_low=3e-7, tau_high=3e-6)
+    run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
+    D = rng.uniform(0.1, 1.0, n_total).astype(np.float32)
+
+    def grad(t):
+        return torch.from_numpy((np.random.default_rng(100 + t).standard_normal(n_total) * 1e-3).astype(np.float32)).cuda()
+
+    assert run.step(1, grad(1), oracle_hz(D, 1, 0, 1), 0) is False
+    cases = [[("g", table[0][0], float("nan"))],
+             [("hz", table[5][0] + 69999, float("inf"))],
+             [("g", table[3][0] + 1, float("-inf")), ("hz", table[2][0], float("nan")), ("g", table[7][0] + 6, float("nan"))],
+             [("g", table[6][0] + 128, float("inf"))]]
+    t = 1
+    for bad in cases:
+        before = (run.w_dev.clone(), run.c_dev.clone(), ta.ta_stats(run.h)[0])
+        t += 1
+        g2, hz = grad(t), oracle_hz(D, 1, 0, t)
+        for which, pos, val in bad:
+            if which == "g":
+                g2[pos] = val
+            else:
+                hz[pos] = val
+        assert run.step(t, g2, hz, 0) is True
+        stats, status = ta.ta_stats(run.h)
+        assert status.skipped == 1 and status.nonfinite_count == len(bad)
+        assert torch.equal(run.w_dev.view(torch.int32), before[0].view(torch.int32)) and torch.equal(run.c_dev, before[1])
+        assert all(a.ema_var == b.ema_var and a.code == b.code and a.lambda_max == b.lambda_max for a, b in zip(stats, before[2]))
+        t += 1
+        assert run.step(t, grad(t), oracle_hz(D, 1, 0, t) if t % 4 else None, 0) is False       # and the pass goes on
+    assert ta.ta_launch_count(run.h) == t          # one launch per step
+
+
 def test_runs_are_bit_reproducible():
     wl = W.get("efficientnet_b0_cifar")
     outs = []
