@@ -1140,8 +1140,8 @@ __global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const F
     // the block's runs folded into one partial per layer it touches, in run order
     cp_async_wait_but_one();        // the block's tables have arrived (the weight copies may still be under way)
     __syncthreads();
-    if (tid < nl) {
-        const uint32_t lo = sh_bl[tid].run_lo, hi = sh_bl[tid].run_hi;
+    for (uint32_t q = tid; q < nl; q += kThreads) {
+        const uint32_t lo = sh_bl[q].run_lo, hi = sh_bl[q].run_hi;
         FusedPartial t{0.0, 0.0, 0u, 0xFFFFFFFFu, 0u, 0u};
         for (uint32_t r = lo; r < hi; ++r) {
             const FusedPartial x = sh_run[r - brun_lo];
@@ -1149,7 +1149,7 @@ __global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const F
             t.amax = max(t.amax, x.amax); t.amin = min(t.amin, x.amin);
             t.bad += x.bad;
         }
-        A.part[bpart_lo + tid] = t;
+        A.part[bpart_lo + q] = t;
     }
 
     if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) {

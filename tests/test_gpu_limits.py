@@ -64,6 +64,33 @@ def test_thousands_of_tiny_layers(ppm, P):
         run.step(t, g, oracle_hz(D, P, 5, t), 5)
 
 
+def test_hundred_thousand_tiny_layers_one_launch():
+    # dense, so the one-launch path: with 120,000 layers of one to three elements a block of its grid touches
+    # several hundred layers (more than it has threads) and a warp walks dozens of runs
+    from paper_2508_16905_b200 import binding as B
+    rng = np.random.default_rng(11)
+    lengths = rng.integers(1, 4, 120000).tolist()
+    table, off = [], 2
+    for j, n in enumerate(lengths):
+        off += int(j % 5 == 0)
+        table.append((off, int(n)))
+        off += int(n)
+    n_total = (off + 7) // 4 * 4
+    runs, used, max_rows = B.ta_plan_one_launch(table, 148 * 24)
+    per_block = {}
+    for _, _, layer, warp in runs:
+        per_block.setdefault(warp // 8, set()).add(layer)
+    assert max(len(v) for v in per_block.values()) > 256
+    hp = dict(beta=0.5, tau_low=3e-7, tau_high=3e-6, tau_curv=0.5, num_probes=1)
+    run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
+    D = np.exp(rng.uniform(np.log(1e-3), 0.0, n_total)).astype(np.float32)
+    for t in (1, 2, 3):
+        g = torch.from_numpy((rng.standard_normal(n_total) * 1e-3).astype(np.float32)).cuda()
+        run.step(t, g, oracle_hz(D, 1, 5, t) if t != 2 else None, 5)
+    if ta.ta_launch_count(run.h) != 3:
+        pytest.skip("this device's grid sent the table to the three-kernel path")
+
+
 @pytest.mark.parametrize("seed", range(40))
 def test_random_tables(seed):
     # random tables, gaps, probe counts, mask fractions and gradient types: planner and kernels against the oracle
