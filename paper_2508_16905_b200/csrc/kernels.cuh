@@ -1654,6 +1654,13 @@ struct ResolveArgs {
     const Status *status;
 };
 
+// Candidate values a thread keeps in flight per pass: one block works on a whole layer, so the passes of a long
+// candidate list are bound by round trips to memory, not by bandwidth.
+#ifndef TA_RESOLVE_LOADS
+#define TA_RESOLVE_LOADS 32
+#endif
+constexpr int kResolveLoads = TA_RESOLVE_LOADS;
+
 // One block per layer: finishes the selection among the layer's candidates.
 __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32_t l)
 {
@@ -1674,12 +1681,12 @@ __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32
 
     // value digits: bits 19..9, then bits 8..0
     clear(kHistBins);
-    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * 8) {
-        uint32_t v[8];
+    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * kResolveLoads) {
+        uint32_t v[kResolveLoads];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { const uint32_t j = j0 + u * kThreads + tid; v[u] = j < m ? __ldg(cv + j) : 0xFFFFFFFFu; }
+        for (int u = 0; u < kResolveLoads; ++u) { const uint32_t j = j0 + u * kThreads + tid; v[u] = j < m ? __ldg(cv + j) : 0xFFFFFFFFu; }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) if (v[u] != 0xFFFFFFFFu) atomicAdd(&h[(v[u] >> 9) & 2047u], 1u);
+        for (int u = 0; u < kResolveLoads; ++u) if (v[u] != 0xFFFFFFFFu) atomicAdd(&h[(v[u] >> 9) & 2047u], 1u);
     }
     __syncthreads();
     block_find_bin<true>(h, kHistBins, s.remaining, scan, found);
@@ -1687,12 +1694,12 @@ __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32
     const uint32_t pre22 = (b1 << 11) | b2;
     __syncthreads();
     clear(512);
-    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * 8) {
-        uint32_t v[8];
+    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * kResolveLoads) {
+        uint32_t v[kResolveLoads];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { const uint32_t j = j0 + u * kThreads + tid; v[u] = j < m ? __ldg(cv + j) : 0xFFFFFFFFu; }
+        for (int u = 0; u < kResolveLoads; ++u) { const uint32_t j = j0 + u * kThreads + tid; v[u] = j < m ? __ldg(cv + j) : 0xFFFFFFFFu; }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) if ((v[u] >> 9) == pre22) atomicAdd(&h[v[u] & 511u], 1u);
+        for (int u = 0; u < kResolveLoads; ++u) if ((v[u] >> 9) == pre22) atomicAdd(&h[v[u] & 511u], 1u);
     }
     __syncthreads();
     block_find_bin<true>(h, 512, r2, scan, found);
@@ -1728,16 +1735,16 @@ __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32
     // set the bits of the taken candidates; their sum is exact: all share sign and exponent
     // (the exponent is part of the level-1 digit), so it is count * 2^e + (sum of mantissas) * 2^(e-23)
     unsigned long long cnt = 0ull, mant = 0ull;
-    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * 8) {
-        uint32_t v[8], ix[8];
+    for (uint32_t j0 = 0; j0 < m; j0 += kThreads * (kResolveLoads / 2)) {
+        uint32_t v[kResolveLoads / 2], ix[kResolveLoads / 2];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kResolveLoads / 2; ++u) {
             const uint32_t j = j0 + u * kThreads + tid;
             v[u] = j < m ? __ldg(cv + j) : 0u;          // 0 is never taken: thr > 0 here or handled by the index rule
             ix[u] = j < m ? __ldg(ci + j) : 0xFFFFFFFFu;
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kResolveLoads / 2; ++u) {
             const uint32_t j = j0 + u * kThreads + tid;
             if (j < m && (v[u] > thr || (v[u] == thr && ix[u] <= idx_limit))) {
                 const uint64_t i = off + ix[u];
