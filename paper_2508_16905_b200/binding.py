@@ -157,7 +157,10 @@ class Handle:
 
     def __del__(self):
         if getattr(self, "ptr", None):
-            lib().ta_destroy(self.ptr)
+            try:
+                lib().ta_destroy(self.ptr)
+            except TypeError:          # interpreter shutdown: the module's globals are already gone
+                pass
             self.ptr = None
 
 
