@@ -40,7 +40,8 @@
 #ifndef TA_APPLY_STREAM_W_STORE
 #define TA_APPLY_STREAM_W_STORE 0
 #endif
-// One-launch path: blocks per SM the compiler must leave room for, slots in flight in the sweep (P <= 1) and in the update.
+// One-launch path: blocks per SM the compiler must leave room for (with one probe or none; two blocks with two or four
+// probes, one with eight, whose rows need more registers), slots in flight in the sweep (P <= 1) and in the update.
 #ifndef TA_FUSED_MIN_BLOCKS
 #define TA_FUSED_MIN_BLOCKS 3
 #endif
@@ -978,7 +979,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsign
 }
 
 template <int P, bool BF16>
-__global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const FusedArgs A)
+__global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <= 4 ? 2 : 1))) k_fused(const FusedArgs A)
 {
     constexpr int PP = P > 0 ? P : 1;
     constexpr int U = (P <= 1) ? TA_FUSED_SWEEP_SLOTS : (P == 2 ? 4 : 2);     // slots in flight per lane during the sweep
@@ -1263,7 +1264,7 @@ __global__ void __launch_bounds__(kThreads, TA_FUSED_MIN_BLOCKS) k_fused(const F
                     x.z = fmaf(neg_eta, gv[u].z, x.z);
                     x.w = fmaf(neg_eta, gv[u].w, x.w);
                     if (e_lo == 0u && e_hi == 4u) {
-                        *reinterpret_cast<float4 *>(A.w + i0) = x;
+                        __stcs(reinterpret_cast<float4 *>(A.w + i0), x);
                         if (code == 0u) {
                             const __half2 a = __floats2half2_rn(x.x, x.y), b = __floats2half2_rn(x.z, x.w);
                             uint2 o;

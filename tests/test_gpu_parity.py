@@ -116,7 +116,7 @@ def ragged_table(lengths, gap_pattern=(0, 1, 3, 5, 0, 7, 2)):
 
 
 @pytest.mark.parametrize("grad_dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("P,ppm", [(1, 1000000), (2, 1000000), (4, 100000), (8, 500000), (1, 1)])
+@pytest.mark.parametrize("P,ppm", [(1, 1000000), (2, 1000000), (4, 1000000), (8, 1000000), (4, 100000), (8, 500000), (1, 1)])
 def test_ragged_segments_odd_offsets(grad_dtype, P, ppm):
     table, n_total = ragged_table(RAGGED)
     rng = np.random.default_rng(P * 7 + ppm % 13)
