@@ -8,3 +8,9 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a)")
+
+
+def pytest_sessionstart(session):
+    """The shared library is built in-tree and not committed: (re)build it when it is missing or older than its sources."""
+    from paper_2508_16905_b200 import build
+    build.build()
