@@ -13,4 +13,8 @@ def pytest_configure(config):
 def pytest_sessionstart(session):
     """The shared library is built in-tree and not committed: (re)build it when it is missing or older than its sources."""
     from paper_2508_16905_b200 import build
-    build.build()
+    try:
+        build.build()
+    except Exception:
+        if not os.path.exists(build.LIB):       # no compiler here and nothing built: the tests that need it say so
+            return
