@@ -32,10 +32,10 @@
 #define TA_SWEEP_MIN_BLOCKS_P4 1
 #endif
 #ifndef TA_APPLY_ROWS
-#define TA_APPLY_ROWS 4
+#define TA_APPLY_ROWS 8
 #endif
 #ifndef TA_APPLY_ROWS_BF16
-#define TA_APPLY_ROWS_BF16 8
+#define TA_APPLY_ROWS_BF16 16
 #endif
 #ifndef TA_APPLY_STREAM_W_STORE
 #define TA_APPLY_STREAM_W_STORE 0
