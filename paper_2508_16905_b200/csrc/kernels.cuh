@@ -732,10 +732,12 @@ __device__ __forceinline__ uint16_t cast16(float x, uint32_t code)
 
 // w <- fl32(w - eta_l g) (Sec. 3.2, Sec. 4.1); c <- RNE cast of the new w for FP16 / BF16 layers (Sec. 2).
 // One batch of the update.  `decision(seg, eta, code)` supplies the layer's step size and precision code.
-template <bool BF16, typename Decision>
+// MOM: the launch has a momentum buffer; its rows are loaded together with the weights and gradients, and fewer rows
+// are kept in flight.
+template <bool BF16, bool MOM, typename Decision>
 __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, const Decision &decision)
 {
-    constexpr int U = BF16 ? TA_APPLY_ROWS_BF16 : TA_APPLY_ROWS;
+    constexpr int U = MOM ? (BF16 ? TA_APPLY_ROWS_BF16 : TA_APPLY_ROWS) / 2 : (BF16 ? TA_APPLY_ROWS_BF16 : TA_APPLY_ROWS);
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     {
         const uint32_t it = batch * kWarps + warp;
@@ -761,9 +763,8 @@ __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, 
                 }
             }
         };
-        auto store_row = [&](uint64_t i0, float4 wv, float4 gv) {
+        auto store_row = [&](uint64_t i0, float4 wv, float4 gv, float4 mv) {
             if (A.mom || A.weight_decay != 0.f) {      // uniform over the launch
-                float4 mv = A.mom ? __ldcs(reinterpret_cast<const float4 *>(A.mom + i0)) : make_float4(0.f, 0.f, 0.f, 0.f);
                 gv.x = sgd_direction(gv.x, wv.x, A.mom ? &mv.x : nullptr, A.momentum, A.weight_decay);
                 gv.y = sgd_direction(gv.y, wv.y, A.mom ? &mv.y : nullptr, A.momentum, A.weight_decay);
                 gv.z = sgd_direction(gv.z, wv.z, A.mom ? &mv.z : nullptr, A.momentum, A.weight_decay);
@@ -799,20 +800,23 @@ __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, 
         if (full_hi > full_lo) {
             uint64_t row = full_lo;
             while (row + U <= full_hi) {
-                float4 wv[U], gv[U];
+                float4 wv[U], gv[U], mv[MOM ? U : 1];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const uint64_t i0 = (row + u) * 128ull + lane * 4u;
                     wv[u] = ld_stream(A.w + i0);
                     gv[u] = GradVec<BF16>::load4(A.g, i0, true);
+                    if (MOM) mv[u] = __ldcs(reinterpret_cast<const float4 *>(A.mom + i0));
                 }
 #pragma unroll
-                for (int u = 0; u < U; ++u) store_row((row + u) * 128ull + lane * 4u, wv[u], gv[u]);
+                for (int u = 0; u < U; ++u)
+                    store_row((row + u) * 128ull + lane * 4u, wv[u], gv[u], MOM ? mv[u] : make_float4(0.f, 0.f, 0.f, 0.f));
                 row += U;
             }
             while (row < full_hi) {
                 const uint64_t i0 = row * 128ull + lane * 4u;
-                store_row(i0, ld_stream(A.w + i0), GradVec<BF16>::load4(A.g, i0, true));
+                store_row(i0, ld_stream(A.w + i0), GradVec<BF16>::load4(A.g, i0, true),
+                          MOM ? __ldcs(reinterpret_cast<const float4 *>(A.mom + i0)) : make_float4(0.f, 0.f, 0.f, 0.f));
                 ++row;
             }
         }
@@ -820,13 +824,13 @@ __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, 
     }
 }
 
-template <bool BF16>
+template <bool BF16, bool MOM>
 __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
 {
     if (A.status->skipped) return;
     const LayerState *state = A.state;
     auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) apply_batch<BF16>(A, batch, decision);
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) apply_batch<BF16, MOM>(A, batch, decision);
 }
 
 // ------------------------------------------------------------------ one launch for small models
@@ -1783,7 +1787,7 @@ __global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
 
 // Top-k steps: the update needs nothing from the resolve step, so both run in ONE launch.  The first
 // n_layers blocks finish the selection of one layer each; the other blocks stride over the update batches.
-template <bool BF16>
+template <bool BF16, bool MOM>
 __global__ void __launch_bounds__(kThreads) k_apply_resolve(const ApplyArgs A, const ResolveArgs R, const uint32_t n_layers)
 {
     if (A.status->skipped) return;
@@ -1794,7 +1798,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_resolve(const ApplyArgs A, c
     const LayerState *state = A.state;
     // eta and code were fixed by k_decide; resolve blocks write other fields (threshold, mass) of the same records
     auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
-    for (uint32_t batch = blockIdx.x - n_layers; batch < A.n_batches; batch += gridDim.x - n_layers) apply_batch<BF16>(A, batch, decision);
+    for (uint32_t batch = blockIdx.x - n_layers; batch < A.n_batches; batch += gridDim.x - n_layers) apply_batch<BF16, MOM>(A, batch, decision);
 }
 
 }  // namespace ta

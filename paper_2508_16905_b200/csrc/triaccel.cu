@@ -177,8 +177,11 @@ void launch_apply(ta_handle *h, float *w, const void *g, uint16_t *c, uint32_t i
     ta::ApplyArgs aa{h->d.items + item_begin, item_count, batches, w, g, c, h->d.state, h->d.status,
                      h->d.mom, h->hp.momentum, h->hp.weight_decay};
     const int grid = (int)std::min<long long>(batches, (long long)h->sm_count * 8);
-    if (h->hp.grad_dtype == TA_GRAD_BF16) ta::k_apply<true><<<grid, ta::kThreads, 0, s>>>(aa);
-    else ta::k_apply<false><<<grid, ta::kThreads, 0, s>>>(aa);
+    const bool bf16 = h->hp.grad_dtype == TA_GRAD_BF16, mom = h->d.mom != nullptr;
+    if (bf16 && mom) ta::k_apply<true, true><<<grid, ta::kThreads, 0, s>>>(aa);
+    else if (bf16) ta::k_apply<true, false><<<grid, ta::kThreads, 0, s>>>(aa);
+    else if (mom) ta::k_apply<false, true><<<grid, ta::kThreads, 0, s>>>(aa);
+    else ta::k_apply<false, false><<<grid, ta::kThreads, 0, s>>>(aa);
     ++h->launches;
 }
 
@@ -774,8 +777,11 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
             if (timed) cudaEventRecord(ev[2], s);
             ta::ApplyArgs aa{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status, d.mom, h->hp.momentum, h->hp.weight_decay};
             const unsigned blocks = (unsigned)h->L + (unsigned)grid;
-            if (bf16) ta::k_apply_resolve<true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-            else ta::k_apply_resolve<false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+            const bool mom = d.mom != nullptr;
+            if (bf16 && mom) ta::k_apply_resolve<true, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+            else if (bf16) ta::k_apply_resolve<true, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+            else if (mom) ta::k_apply_resolve<false, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+            else ta::k_apply_resolve<false, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
             h->launches += 2;
             if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
             TA_CUDA(h, cudaGetLastError());
