@@ -10,6 +10,9 @@ Tolerances (the bar the method's specification sets):
   mean, EMA mean           1e-5 * max(|mean|, sqrt(var + mean^2))
   master weights           <= 2 ulp (float);  16-bit copies <= 1 ulp of their format
 """
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import torch
 
@@ -75,16 +78,66 @@ def compare_stats(gl, ol, where=""):
     return near
 
 
+class ShardedOracle:
+    """Several oracle instances, each over a share of the layers, stepped on one host thread each (layers are
+    independent and the C call releases the interpreter lock), behind the interface of one oracle.  Only for
+    finite inputs: a step that one share would skip is a whole-step skip for a single oracle, so it is refused here."""
+
+    def __init__(self, table, n_total, threads, **hp):
+        order = sorted(range(len(table)), key=lambda j: -table[j][1])
+        shares, load = [[] for _ in range(max(1, min(threads, len(table))))], [0] * max(1, min(threads, len(table)))
+        for j in order:                                   # longest layer first, to the least loaded share
+            k = load.index(min(load))
+            shares[k].append(j)
+            load[k] += table[j][1]
+        self.shares = [sorted(sh) for sh in shares if sh]
+        self.parts = [orc.Oracle([table[j] for j in sh], n_total, **hp) for sh in self.shares]
+        self.where = {j: (k, i) for k, sh in enumerate(self.shares) for i, j in enumerate(sh)}
+        self.n_layers = len(table)
+        self.pool = ThreadPoolExecutor(len(self.parts))
+
+    def set_lr(self, eta0):
+        for o in self.parts:
+            o.set_lr(eta0)
+
+    def step(self, w, g, hz, c, seed, t):
+        skipped = list(self.pool.map(lambda o: o.step(w, g, hz, c, seed, t), self.parts))
+        assert not any(skipped), "sharded oracle: non-finite input (use a single oracle for skip semantics)"
+        return False
+
+    def layers(self):
+        per = [o.layers() for o in self.parts]
+        return [per[self.where[j][0]][self.where[j][1]] for j in range(self.n_layers)]
+
+    def status(self):
+        st = [o.status() for o in self.parts]
+        out = st[0]
+        out.nonfinite_count = sum(s.nonfinite_count for s in st)
+        out.near_threshold_count = sum(s.near_threshold_count for s in st)
+        return out
+
+    def mask(self):
+        m = self.parts[0].mask()
+        for o in self.parts[1:]:
+            m |= o.mask()
+        return m
+
+    def codes(self):
+        return np.array([ly.code for ly in self.layers()], dtype=np.uint8)
+
+
 class ParityRun:
     """One workload on both sides.  `layers` restricts the oracle (and the comparison) to a subset of
     the layers: layers are independent, so the oracle of a subset equals the full oracle on that subset."""
 
-    def __init__(self, table, n_total, hp, w0, layers=None):
+    def __init__(self, table, n_total, hp, w0, layers=None, threads=1):
         self.table, self.n_total, self.hp = list(table), int(n_total), dict(hp)
         self.layers = list(range(len(table))) if layers is None else list(layers)
         self.sub_table = [self.table[l] for l in self.layers]
         self.h = ta.ta_create(self.table, self.n_total, **self.hp)
-        self.o = orc.Oracle(self.sub_table, self.n_total, **self.hp)
+        threads = min(int(threads), os.cpu_count() or 1)
+        self.o = (orc.Oracle(self.sub_table, self.n_total, **self.hp) if threads <= 1 else
+                  ShardedOracle(self.sub_table, self.n_total, threads, **self.hp))
         self.w_dev = w0.to("cuda").clone()
         self.c_dev = torch.full((self.n_total,), 0x5A5A, dtype=torch.int16, device="cuda")
         self.w_host = to_host_bits(w0).copy()
@@ -93,6 +146,7 @@ class ParityRun:
         self.inside_all = segment_mask(self.table, self.n_total)
         self.inside_sub = segment_mask(self.sub_table, self.n_total)
         self.near_list = []
+        self.layer_steps = 0
         self.max_w_ulp = 0
         self.max_c_ulp = 0
 
@@ -115,6 +169,7 @@ class ParityRun:
         olayers = self.o.layers()
         codes_gpu = ta.ta_precision_codes(self.h)
         near_now = set()
+        self.layer_steps += len(self.layers)
         for j, l in enumerate(self.layers):
             if compare_stats(stats[l], olayers[j], where=f"step {t} layer {l}"):
                 near_now.add(l)
@@ -155,3 +210,12 @@ class ParityRun:
                 assert np.array_equal(bg, bo)
         else:
             assert ta.ta_masks(self.h) == (None, 0)
+
+    def report(self, name, max_fraction=0.01):
+        """Lists the near-threshold exceptions of the run (layer-steps where either side flagged a statistic within
+        1e-5 relative of a decision threshold, the only place where codes may differ) and bounds their number."""
+        print(f"{name}: {self.layer_steps} layer-steps compared, {len(self.near_list)} near a threshold; "
+              f"max distance master weights {self.max_w_ulp} ulp, 16-bit copies {self.max_c_ulp} ulp")
+        for t, l, code_gpu, code_oracle in self.near_list:
+            print(f"  near threshold: step {t} layer {l} code gpu {code_gpu} oracle {code_oracle}")
+        assert len(self.near_list) <= max(1, int(max_fraction * self.layer_steps)), "too many near-threshold layer-steps"

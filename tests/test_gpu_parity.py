@@ -11,14 +11,15 @@ from tests.parity import ParityRun, oracle_hz, to_host_bits, ulp_f32, ulp_16
 pytestmark = pytest.mark.gpu
 
 
-def run_workload(wl, steps, hz_every=1, layers=None, check_every=1):
+def run_workload(wl, steps, hz_every=1, layers=None, check_every=1, threads=1):
     w0 = W.make_weights(wl, "cuda")
     D = W.make_curvature(wl, "cuda").cpu().numpy()
-    run = ParityRun(wl.table, wl.n_total, wl.hparams(), w0, layers=layers)
+    run = ParityRun(wl.table, wl.n_total, wl.hparams(), w0, layers=layers, threads=threads)
     for t in range(1, steps + 1):
         g = W.make_grads(wl, t, "cuda")
         hz = oracle_hz(D, wl.num_probes, wl.probe_seed, t) if (t - 1) % hz_every == 0 else None
         run.step(t, g, hz, wl.probe_seed, check=(t % check_every == 0 or t == steps))
+    run.report(wl.name)
     return run
 
 
@@ -61,40 +62,48 @@ def test_efficientnet_b0_unpadded_offsets():
     run_workload(W.get("efficientnet_b0_cifar", align=1), 3)
 
 
-def test_resnet50_topk_full_size():
+def test_resnet50_topk_full_size_all_steps():
+    # all 50 steps at full size; the oracle runs one instance per host thread over a share of the layers
     wl = W.get("resnet50_topk")
-    run_workload(wl, 3)
+    run_workload(wl, wl.steps, check_every=5, threads=8)
 
 
-def test_resnet50_topk_quarter_width_all_steps():
+def test_resnet50_topk_quarter_width_curvature_every_third_step():
     wl = W.get("resnet50_topk", shapes=W.resnet50_shapes(width=16))
-    run_workload(wl, wl.steps, check_every=5)
+    run_workload(wl, 12, hz_every=3, check_every=2)
 
 
-def test_gpt_1p3b_sampled_layers():
-    # full-size run on the GPU; the oracle follows a sample of layers (independent of the rest):
-    # the embedding, the first block, and the last block
+def test_gpt_1p3b_all_steps_sampled_layers():
+    # full-size run on the GPU for all 20 steps; the oracle follows a sample of layers (independent of the rest):
+    # the embedding, the first block, a middle block and the last block.  Curvature arrives on every fourth step
+    # only, so that lambda_l is held over between refreshes at full size.
     wl = W.get("gpt_1p3b")
     L = len(wl.table)
-    layers = list(range(0, 7)) + list(range(L - 6, L))
+    mid = 1 + 6 * 12
+    layers = list(range(0, 7)) + list(range(mid, mid + 6)) + list(range(L - 6, L))
     w0 = W.make_weights(wl, "cuda")
     D_dev = W.make_curvature(wl, "cuda")
-    run = ParityRun(wl.table, wl.n_total, wl.hparams(), w0, layers=layers)
+    D_host = {l: D_dev[wl.table[l][0]:wl.table[l][0] + wl.table[l][1]].cpu().numpy() for l in layers}
+    run = ParityRun(wl.table, wl.n_total, wl.hparams(), w0, layers=layers, threads=8)
     del w0
     z = torch.empty(wl.n_total, device="cuda")
-    for t in (1, 2):
+    for t in range(1, wl.steps + 1):
         g = W.make_grads(wl, t, "cuda")
-        ta.ta_probe(run.h, wl.probe_seed, t, 0, z)
-        hz_dev = D_dev * z
-        # oracle-side Hz is built from the oracle's own probe on the sampled layers, and only there
-        hz_host = np.zeros(wl.n_total, dtype=np.float32)
-        for l in layers:
-            off, n = wl.table[l]
-            zo = orc.probe(wl.probe_seed, t, 0, off, n)
-            assert np.array_equal(zo, z[off:off + n].cpu().numpy())
-            hz_host[off:off + n] = D_dev[off:off + n].cpu().numpy() * zo
-        run.step(t, g, hz_host, wl.probe_seed, hz_dev=hz_dev)
+        hz_dev = hz_host = None
+        if (t - 1) % 4 == 0:
+            ta.ta_probe(run.h, wl.probe_seed, t, 0, z)
+            hz_dev = D_dev * z
+            # oracle-side Hz is built from the oracle's own probe on the sampled layers, and only there
+            hz_host = np.zeros(wl.n_total, dtype=np.float32)
+            for l in layers:
+                off, n = wl.table[l]
+                zo = orc.probe(wl.probe_seed, t, 0, off, n)
+                if t == 1:
+                    assert np.array_equal(zo, z[off:off + n].cpu().numpy())
+                hz_host[off:off + n] = D_host[l] * zo
+        run.step(t, g, hz_host, wl.probe_seed, hz_dev=hz_dev, check=(t in (1, 2, 5, 10, 15, 20)))
         del hz_dev, hz_host, g
+    run.report(wl.name + " (19 of 145 layers)")
     # every layer, not only the sampled ones, must have produced finite statistics and a code
     stats, status = ta.ta_stats(run.h)
     assert status.skipped == 0 and status.nonfinite_count == 0
