@@ -207,7 +207,7 @@ def run_ours(args):
     torch.cuda.set_device(local_rank if world > 1 else 0)
     dev = torch.device("cuda", torch.cuda.current_device())
     props = torch.cuda.get_device_properties(dev)
-    wl = W.get(args.config)
+    wl = W.get(args.config, **({"t_ctrl": args.t_ctrl} if args.t_ctrl else {}))
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     P, N = wl.num_probes, wl.n_total
     l2_bytes = props.L2_cache_size
@@ -216,7 +216,7 @@ def run_ours(args):
     state_bytes = N * 6
     # rotate over R buffer sets so that consecutive steps never find their inputs in L2
     R = 1 if (bytes_in_per_set + state_bytes) > 4 * l2_bytes else max(2, -(-6 * l2_bytes // (bytes_in_per_set + state_bytes)))
-    hp = dict(wl.hparams(), momentum=args.momentum, weight_decay=args.weight_decay)
+    hp = dict(wl.hparams(), momentum=args.momentum, weight_decay=args.weight_decay, flags=1 if args.inputs_finite else 0)
     h = ta.ta_create(wl.table, N, **hp)
     curv = W.make_curvature(wl, dev)
     sets = []
@@ -406,6 +406,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--momentum", type=float, default=0.0)
     ap.add_argument("--weight-decay", type=float, default=0.0)
+    ap.add_argument("--t-ctrl", type=int, default=0, help="override the workload's control interval T_ctrl")
+    ap.add_argument("--inputs-finite", action="store_true", help="create the handle with TA_FLAG_INPUTS_FINITE")
     ap.add_argument("--op", default="step", choices=["step", "power"], help="step: the optimizer pass (default); power: ta_power_iterate")
     ap.add_argument("--deflate", type=int, default=0, help="--op power: number of deflated eigenvectors")
     args = ap.parse_args()

@@ -80,8 +80,31 @@ typedef struct {
     uint32_t grad_dtype; /* TA_GRAD_F32 or TA_GRAD_BF16 */
     float momentum;      /* SGD momentum mu in [0,1); 0 = plain SGD               Sec. 4.1 */
     float weight_decay;  /* L2 coefficient wd >= 0 added to the gradient; 0 = none       */
-    uint32_t flags;      /* must be 0 */
+    uint32_t flags;      /* 0 or TA_FLAG_* bits */
 } ta_hparams;
+
+/*
+ * TA_FLAG_INPUTS_FINITE -- the caller vouches that g and Hz hold no inf / NaN inside the segments (a mixed-precision
+ * loop knows this from its own overflow check when it unscales the gradients).  Without the flag, one non-finite value
+ * anywhere makes the whole step change nothing, so no layer can be updated before every layer has been read once, and
+ * the gradient is read from memory twice.  With the flag the pass no longer holds the update back:
+ *   - at a step with decisions (step % t_ctrl == 0) every layer is updated as soon as its own statistics are complete
+ *     (Sec. 3.1, 3.2: all decisions are per layer), while its gradient is still in the L2 cache;
+ *   - at a step without decisions (Sec. 3.4) the step size and the code of every layer are known beforehand, and the
+ *     statistics, the update and the cast run as a single pass that reads every input once.
+ * On finite inputs the results are those of the default pass.  Non-finite values are still counted
+ * (ta_step_status.nonfinite_count) but no longer stop the step: skipped stays 0 and the layers that held them carry
+ * non-finite statistics and weights.  Used by large dense models (no top-k mask, no momentum, beyond the size of the
+ * one-launch path); other handles accept the flag and run the default pass.
+ */
+#define TA_FLAG_INPUTS_FINITE 1u
+/*
+ * TA_FLAG_NO_ONE_LAUNCH -- small dense models normally run the whole pass as one cooperative launch; with this flag
+ * the handle uses the kernels of large models instead (separate sweep / decide / update launches, or the pipelined
+ * launch together with TA_FLAG_INPUTS_FINITE).  Results are the same; meant for diagnostics and for exercising those
+ * kernels on small tables.
+ */
+#define TA_FLAG_NO_ONE_LAUNCH 2u
 
 /* Per-layer statistics as of the last ta_step (host side, filled by ta_stats). */
 typedef struct {
@@ -263,6 +286,28 @@ typedef struct ta_run {
 int ta_plan_one_launch(const ta_segment *table, uint32_t L, uint32_t warps, ta_run *out, uint32_t cap,
                        uint32_t *n_runs, uint32_t *warps_used, uint32_t *max_rows);
 
+/*
+ * The task queues of the pipelined pass (TA_FLAG_INPUTS_FINITE on a large dense model), for inspection (host only,
+ * no GPU needed).  Every task covers one batch: up to 14336 consecutive elements of one layer.  With
+ * with_decisions != 0, the two queues of a step that takes decisions (Sec. 3.4), one after the other: the sweep tasks
+ * (TA_TASK_SWEEP, statistics) in buffer order, then the update tasks (TA_TASK_APPLY) layer by layer, within a layer
+ * the last batch first.  Blocks draw from both queues; an update task is handed out once its layer is decided, and
+ * until then the block goes on sweeping.  Otherwise the queue of a step between decisions, one single-pass task
+ * (TA_TASK_BOTH) per batch.  Writes at most cap tasks; *n_tasks is their number (TA_ERR_ARG if cap is smaller).
+ * Table rules as for ta_create.
+ */
+#define TA_TASK_SWEEP 0u
+#define TA_TASK_APPLY 1u
+#define TA_TASK_BOTH  2u
+typedef struct ta_task {
+    uint64_t begin;      /* first element of the batch */
+    uint32_t length;     /* elements, all inside one layer */
+    uint32_t layer;
+    uint32_t kind;       /* TA_TASK_* */
+    uint32_t reserved;
+} ta_task;
+int ta_plan_pipeline(const ta_segment *table, uint32_t L, uint32_t with_decisions, ta_task *out, uint64_t cap, uint64_t *n_tasks);
+
 /* Static description of the last error of this handle ("" if none).  h may be NULL: then the
  * last ta_create failure of the calling thread. */
 const char *ta_last_error(const ta_handle *h);
@@ -313,23 +358,29 @@ int ta_batch_next(ta_batch_ctrl *bc, int64_t *B_next);
  * whose memory pool was sized up front and must not grow.  ta_create / ta_step allocate their
  * workspace with cudaMalloc; this call never calls cudaMalloc, cudaFree or any allocating routine.
  *
- * How: the scratch (one partial sum, sum of squares and non-finite count per tile of
- * TA_STATIC_TILE_ELEMS gradient elements) lives in a fixed array inside the library's device
- * image, about 640 KB, which every GPU that loads the library holds until the process exits.
- * The layer table travels as a kernel argument.
+ * How: the scratch (per tile of TA_STATIC_TILE_ELEMS gradient elements: two partial sums, the tile's
+ * pivot value and a non-finite count) lives in a fixed array inside the library's device image, about
+ * 770 KB.  A GPU holds it from the moment the CUDA runtime loads this library's device code there until
+ * the process exits.  The layer table travels as a kernel argument.
+ *
+ * The first call on each device is a warm-up: with the CUDA runtime's default lazy loading it is that
+ * call which loads the device code (kernels and the array) onto the device, which takes device memory
+ * once and can fail when none is left, and it looks up the array's device address (cudaGetSymbolAddress,
+ * with that device current).  Make it at start-up, while memory is still free, outside any stream
+ * capture and outside allocator locks (or run with CUDA_MODULE_LOADING=EAGER, which moves the loading
+ * to context creation).  Every later call on that device allocates nothing at all: free device memory
+ * is the same before and after it.
  *
  *   table      host, L <= TA_STATIC_MAX_LAYERS segments, same rules as ta_create
  *   g          device, float or bfloat16 per grad_dtype, 16-byte aligned, indexed by flat element
  *   mean_var   device double[2 * L] (output): mean of layer l at [2l], variance at [2l + 1]
- *   nonfinite  device uint32[L] (output) or NULL: non-finite gradient values per layer
+ *   nonfinite  device uint32[L] (output, 4-byte aligned) or NULL: non-finite gradient values per layer
  *   stream     cudaStream_t as void*; the call is asynchronous
  *
  * Limits: the layers must fit in TA_STATIC_MAX_TILES tiles (tiles are cut on a global grid of
  * TA_STATIC_TILE_ELEMS elements, so a layer of n elements needs about n / TA_STATIC_TILE_ELEMS + 1);
  * that is roughly 536 million parameters.  A larger table is rejected with TA_ERR_ARG and a message
  * (ta_static_last_error) and nothing is launched.
- * The first call on each device looks up the device address of the array (cudaGetSymbolAddress, with
- * that device current); make that first call outside any stream capture.
  * All calls on one device share the one array and it keeps the previous call's contents.  Every
  * slot a call reads is written earlier in the same call, so nothing needs clearing; but two calls
  * whose kernels overlap on the GPU (different streams, no ordering between them) race on it and

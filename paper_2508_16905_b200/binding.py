@@ -16,12 +16,13 @@ LIB_PATH = os.path.join(HERE, "libtriaccel.so")
 TA_OK, TA_ERR_ARG, TA_ERR_ALIGN, TA_ERR_STATE, TA_ERR_CUDA, TA_ERR_NOMEM = 0, -1, -2, -3, -4, -5
 TA_CODE_FP16, TA_CODE_BF16, TA_CODE_FP32 = 0, 1, 2
 TA_GRAD_F32, TA_GRAD_BF16 = 0, 1
+TA_FLAG_INPUTS_FINITE, TA_FLAG_NO_ONE_LAUNCH = 1, 2
 
 EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "ta_probe", "ta_stats",
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
            "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
            "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait",
-           "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch"]
+           "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch", "ta_plan_pipeline"]
 
 
 class ta_segment(C.Structure):
@@ -30,6 +31,11 @@ class ta_segment(C.Structure):
 
 class ta_run(C.Structure):
     _fields_ = [("begin", C.c_uint64), ("length", C.c_uint32), ("layer", C.c_uint32), ("warp", C.c_uint32),
+                ("reserved", C.c_uint32)]
+
+
+class ta_task(C.Structure):
+    _fields_ = [("begin", C.c_uint64), ("length", C.c_uint32), ("layer", C.c_uint32), ("kind", C.c_uint32),
                 ("reserved", C.c_uint32)]
 
 
@@ -103,6 +109,7 @@ def lib():
     L.ta_set_curvature.argtypes = [vp, vp]
     L.ta_plan_one_launch.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_run), u32, C.POINTER(u32), C.POINTER(u32),
                                      C.POINTER(u32)]
+    L.ta_plan_pipeline.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_task), u64, C.POINTER(u64)]
     L.ta_static_last_error.argtypes = []
     L.ta_static_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -291,6 +298,21 @@ def ta_plan_one_launch(table, warps):
     if rc != TA_OK:
         raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
     return [(r.begin, r.length, r.layer, r.warp) for r in out[:n.value]], used.value, rows.value
+
+
+def ta_plan_pipeline(table, with_decisions=True):
+    """The task queue of the pipelined pass as a list of (kind, layer, begin, length); kind 0 sweep, 1 apply, 2 both."""
+    L = len(table)
+    segs = (ta_segment * max(L, 1))(*[ta_segment(int(o), int(n)) for o, n in table])
+    n = C.c_uint64()
+    rc = lib().ta_plan_pipeline(segs, L, 1 if with_decisions else 0, None, 0, C.byref(n))
+    if rc != TA_OK and n.value == 0:
+        raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
+    out = (ta_task * max(1, n.value))()
+    rc = lib().ta_plan_pipeline(segs, L, 1 if with_decisions else 0, out, n.value, C.byref(n))
+    if rc != TA_OK:
+        raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
+    return [(t.kind, t.layer, t.begin, t.length) for t in out[:n.value]]
 
 
 def ta_test_expire_next_wait(h):

@@ -29,7 +29,7 @@
 #define TA_SWEEP_ROWS_P4 2
 #endif
 #ifndef TA_SWEEP_MIN_BLOCKS_P4
-#define TA_SWEEP_MIN_BLOCKS_P4 1
+#define TA_SWEEP_MIN_BLOCKS_P4 2
 #endif
 #ifndef TA_APPLY_ROWS
 #define TA_APPLY_ROWS 8
@@ -238,8 +238,11 @@ struct SweepArgs {
     uint64_t n_total;
     uint64_t seed;
     uint32_t step;
-    // per-item partial results
+    // per-item partial results; p_s1 / p_s2 are sums of (x - pivot) and (x - pivot)^2, the pivot being the item's
+    // first gradient value (p_piv): the variance of a layer whose mean is far larger than its spread then comes out
+    // of numbers of the size of the spread instead of the difference of two nearly equal sums
     double *p_s1, *p_s2, *p_sa;
+    float *p_piv;
     uint32_t *p_amax, *p_amin, *p_bad;
     // top-k only
     float *abs_s;             // [n_total] |S|
@@ -252,6 +255,48 @@ constexpr uint32_t kMixedBatch = 0xFFFFFFFFu;
 template <int P> struct RowData {
     float4 g;
     float4 hz[P > 0 ? P : 1];
+    float4 w;                 // only used by the single-pass variant of the sweep
+};
+
+// w <- fl32(w - eta g) for one 16-byte vector, stored together with its 16-bit cast when the layer keeps a copy
+// (code 0: binary16, 1: bfloat16, 2: none).  Sec. 3.2 step, Sec. 2 master copy and cast.
+template <bool STREAM_W>
+__device__ __forceinline__ void update_store4(float *w, uint16_t *c, uint64_t i0, float4 wv, const float4 gv, float neg_eta, uint32_t code)
+{
+    wv.x = fmaf(neg_eta, gv.x, wv.x);
+    wv.y = fmaf(neg_eta, gv.y, wv.y);
+    wv.z = fmaf(neg_eta, gv.z, wv.z);
+    wv.w = fmaf(neg_eta, gv.w, wv.w);
+    if (STREAM_W) __stcs(reinterpret_cast<float4 *>(w + i0), wv);
+    else *reinterpret_cast<float4 *>(w + i0) = wv;
+    if (code == 0u) {
+        const __half2 a = __floats2half2_rn(wv.x, wv.y), b = __floats2half2_rn(wv.z, wv.w);
+        uint2 o;
+        o.x = *reinterpret_cast<const uint32_t *>(&a);
+        o.y = *reinterpret_cast<const uint32_t *>(&b);
+        __stcs(reinterpret_cast<uint2 *>(c + i0), o);
+    } else if (code == 1u) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(wv.x, wv.y), b = __floats2bfloat162_rn(wv.z, wv.w);
+        uint2 o;
+        o.x = *reinterpret_cast<const uint32_t *>(&a);
+        o.y = *reinterpret_cast<const uint32_t *>(&b);
+        __stcs(reinterpret_cast<uint2 *>(c + i0), o);
+    }
+}
+
+__device__ __forceinline__ uint16_t cast16(float x, uint32_t code)
+{
+    return code == 0u ? __half_as_ushort(__float2half_rn(x)) : __bfloat16_as_ushort(__float2bfloat16_rn(x));
+}
+
+// What the single-pass variant of the sweep needs besides the sweep's own arguments: on a step without decisions the
+// step size and the precision code of every layer are known beforehand (Sec. 3.4: decisions only every T_ctrl steps),
+// so the update can be applied in the pass that gathers the statistics.
+struct SinglePass {
+    float *w;
+    uint16_t *c;
+    const LayerState *state;
+    float eta0;
 };
 
 // Balanced pairwise sum: adjacent pairs, level by level.
@@ -270,6 +315,7 @@ template <int P> __device__ __forceinline__ float pairwise(const float (&t)[P > 
 }
 
 template <int P, bool TOPK> struct SweepAcc {
+    double pivot = 0.0;     // subtracted from every gradient value before it is summed
     double s1 = 0.0, s2 = 0.0, sa = 0.0;
     float sa_row = 0.f;     // |S| of the current row (four values), folded into sa by end_row()
     uint32_t amax = 0u, amin = 0xFFFFFFFFu, gmax = 0u;
@@ -282,7 +328,7 @@ template <int P, bool TOPK> struct SweepAcc {
     {
         const uint32_t gb = __float_as_uint(gv) & 0x7FFFFFFFu;
         gmax = max(gmax, gb);
-        const double x = (double)gv;
+        const double x = (double)gv - pivot;
         s1 += x;
         s2 = fma(x, x, s2);
         uint32_t ab = 0u;
@@ -306,12 +352,23 @@ template <int P, bool TOPK> struct SweepAcc {
     }
 };
 
-// One batch (eight items, one per warp) of the sweep.  Called by the whole block.
-template <int P, bool BF16, bool TOPK>
-__device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, uint32_t *sh_hist)
+// What one item contributes to its layer's statistics (valid in lane 0 of the warp that swept it).
+struct ItemSums {
+    double s1, s2, sa;           // sums of (g - piv), (g - piv)^2 and |S|
+    float piv;
+    uint32_t n, amax, amin, bad;
+};
+
+// One batch (eight items, one per warp) of the sweep.  Called by the whole block.  `store(it, sums)` is called by
+// lane 0 of each warp with the results of item `it`.  APPLY: the single-pass variant, which also updates the weights
+// of the rows it sweeps (with the step size and code the layers had before this step) and writes their 16-bit copies.
+template <int P, bool BF16, bool TOPK, bool APPLY, int ROWS = 0, typename Store>
+__device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, uint32_t *sh_hist, const Store &store,
+                                            const SinglePass &sp = SinglePass{nullptr, nullptr, nullptr, 0.f})
 {
+    static_assert(!(APPLY && TOPK), "the single-pass variant is for dense curvature");
     constexpr int PP = P > 0 ? P : 1;
-    constexpr int U = (P <= 1) ? (BF16 ? TA_SWEEP_ROWS_P1_BF16 : TA_SWEEP_ROWS_P1)
+    constexpr int U = ROWS > 0 ? ROWS : (P <= 1) ? (BF16 ? TA_SWEEP_ROWS_P1_BF16 : TA_SWEEP_ROWS_P1)
                                : (P == 2 ? TA_SWEEP_ROWS_P2 : TA_SWEEP_ROWS_P4);     // rows in flight per lane
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     {
@@ -327,15 +384,20 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             __syncthreads();
         }
         const Item item = it < A.n_items ? A.items[it] : Item{0, 0, 0};
-        if (it < A.n_items && item.len == 0u && lane == 0) {   // padding item: neutral partials
-            A.p_s1[it] = 0.0; A.p_s2[it] = 0.0; A.p_bad[it] = 0u;
-            if (P > 0) { A.p_amax[it] = 0u; A.p_amin[it] = 0xFFFFFFFFu; }
-            if (TOPK) A.p_sa[it] = 0.0;
-        }
+        if (it < A.n_items && item.len == 0u && lane == 0)     // padding item: neutral partials
+            store(it, ItemSums{0.0, 0.0, 0.0, 0.f, 0u, 0u, 0xFFFFFFFFu, 0u});
         if (item.len != 0u) {
         const uint64_t begin = item.begin, end = begin + item.len;
         const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
         SweepAcc<P, TOPK> acc;
+        const float piv = GradVec<BF16>::load1(A.g, begin);
+        acc.pivot = (double)piv;
+        float neg_eta = 0.f;
+        uint32_t code = 2u;
+        if (APPLY) {
+            neg_eta = -__fmul_rn(sp.eta0, sp.state[item.seg].eta_scale);
+            code = sp.state[item.seg].code;
+        }
         auto hist_add = [&](uint32_t ab) {
             if (uniform) atomicAdd(&sh_hist[ab >> 20], 1u);
             else atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
@@ -369,7 +431,13 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                     float hv[PP];
 #pragma unroll
                     for (int p = 0; p < PP; ++p) hv[p] = (P > 0) ? __ldcs(A.hz + (uint64_t)p * A.n_total + i) : 0.f;
-                    const uint32_t ab = acc.element(GradVec<BF16>::load1(A.g, i), hv, sel, (k & 7u) * 4u + e);
+                    const float gv = GradVec<BF16>::load1(A.g, i);
+                    const uint32_t ab = acc.element(gv, hv, sel, (k & 7u) * 4u + e);
+                    if (APPLY) {
+                        const float wn = fmaf(neg_eta, gv, sp.w[i]);
+                        sp.w[i] = wn;
+                        if (code < 2u) sp.c[i] = cast16(wn, code);
+                    }
                     if (TOPK) {
                         A.abs_s[i] = __uint_as_float(ab);
                         hist_add(ab);
@@ -406,6 +474,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                         const uint64_t i0 = (row + u) * 128ull + lane * 4u;
                         *reinterpret_cast<float4 *>(A.abs_s + i0) = make_float4(av[0], av[1], av[2], av[3]);
                     }
+                    if (APPLY) update_store4<true>(sp.w, sp.c, (row + u) * 128ull + lane * 4u, rd[u].w, rd[u].g, neg_eta, code);
                 }
             }
         };
@@ -415,10 +484,11 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             for (int u = 0; u < U; ++u) {
                 if (u < count) {
                     const uint64_t i0 = (row + u) * 128ull + lane * 4u;
-                    rd[u].g = GradVec<BF16>::load4(A.g, i0, false);
+                    rd[u].g = GradVec<BF16>::load4(A.g, i0, APPLY);       // read once when the update rides along
 #pragma unroll
                     for (int p = 0; p < PP; ++p)
                         if (P > 0) rd[u].hz[p] = ld_stream(A.hz + (uint64_t)p * A.n_total + i0);
+                    if (APPLY) rd[u].w = ld_stream(sp.w + i0);
                 }
             }
         };
@@ -472,13 +542,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             }
             bad = __reduce_add_sync(0xFFFFFFFFu, bad);
         }
-        if (lane == 0) {
-            A.p_s1[it] = s1;
-            A.p_s2[it] = s2;
-            A.p_bad[it] = bad;
-            if (P > 0) { A.p_amax[it] = amax; A.p_amin[it] = amin; }
-            if (TOPK) A.p_sa[it] = sa;
-        }
+        if (lane == 0) store(it, ItemSums{s1, s2, sa, piv, item.len, amax, amin, bad});
         }   // item.len != 0
         if (TOPK) {
             __syncthreads();
@@ -493,13 +557,30 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
 }
 
 template <int P, bool BF16, bool TOPK>
-__global__ void __launch_bounds__(kThreads, (P >= 4 ? TA_SWEEP_MIN_BLOCKS_P4 : 1)) k_sweep(const SweepArgs A)
+__global__ void __launch_bounds__(kThreads, (P == 4 ? TA_SWEEP_MIN_BLOCKS_P4 : 1)) k_sweep(const SweepArgs A)
 {
     __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK>(A, batch, sh_hist);
+    auto store = [&A](uint32_t it, const ItemSums &r) {
+        A.p_s1[it] = r.s1;
+        A.p_s2[it] = r.s2;
+        A.p_piv[it] = r.piv;
+        A.p_bad[it] = r.bad;
+        if (P > 0) { A.p_amax[it] = r.amax; A.p_amin[it] = r.amin; }
+        if (TOPK) A.p_sa[it] = r.sa;
+    };
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK, false>(A, batch, sh_hist, store);
 }
 
 // ------------------------------------------------------------------ decisions
+
+// Sums of (x - p) and (x - p)^2 over n values, moved from pivot p to pivot q:  with d = p - q,
+//   sum (x - q) = s1 + n d,   sum (x - q)^2 = s2 + d (2 s1 + n d).
+struct MomentSums { double s1, s2; };
+__device__ __forceinline__ MomentSums rebase(double s1, double s2, double n, double p, double q)
+{
+    const double d = p - q;
+    return MomentSums{fma(n, d, s1), fma(d, fma(n, d, 2.0 * s1), s2)};
+}
 
 // Whole block: the bin in which the `need`-th element falls when bins are walked from the top
 // (DESC) or from the bottom, and how many elements lie in the bins walked before it.
@@ -539,7 +620,9 @@ __device__ __forceinline__ void block_find_bin(const uint32_t *h, int bins, uint
 struct DecideArgs {
     const uint32_t *item_lo;        // [L + 1] first item of each layer
     const uint64_t *seg_len;        // [L]
+    const Item *items;
     const double *p_s1, *p_s2, *p_sa;
+    const float *p_piv;
     const uint32_t *p_amax, *p_amin, *p_bad;
     LayerScratch *scratch;          // [L]
     LayerState *state;              // [L]
@@ -648,10 +731,13 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     }
     double s1 = 0.0, s2 = 0.0, sa = 0.0, bad = 0.0;
     uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+    // every item summed around its own pivot; here the sums are moved to the pivot of the layer's first item
+    const double pivot = (double)A.p_piv[lo];
 #pragma unroll 4
     for (uint32_t i = lo + tid; i < hi; i += kThreads) {
-        s1 += A.p_s1[i];
-        s2 += A.p_s2[i];
+        const MomentSums m = rebase(A.p_s1[i], A.p_s2[i], (double)A.items[i].len, (double)A.p_piv[i], pivot);
+        s1 += m.s1;
+        s2 += m.s2;
         bad += (double)A.p_bad[i];
         if (A.has_hz) {
             amax = max(amax, A.p_amax[i]);
@@ -670,11 +756,11 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     if (tid == 0) {
         for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
         const double n = (double)A.seg_len[l];
-        const double mu = s1 / n;
-        double var = s2 / n - mu * mu;
+        const double shift = s1 / n;
+        double var = s2 / n - shift * shift;
         if (!(var > 0.0)) var = 0.0;
         LayerScratch sc;
-        sc.mean = mu; sc.var = var; sc.sum_abs = sa;
+        sc.mean = pivot + shift; sc.var = var; sc.sum_abs = sa;
         sc.bad = (unsigned long long)bad;
         sc.amax = amax; sc.amin = amin;
         A.scratch[l] = sc;
@@ -725,19 +811,18 @@ __device__ __forceinline__ float sgd_direction(float g, float w, float *buf, flo
     return d;
 }
 
-__device__ __forceinline__ uint16_t cast16(float x, uint32_t code)
-{
-    return code == 0u ? __half_as_ushort(__float2half_rn(x)) : __bfloat16_as_ushort(__float2bfloat16_rn(x));
-}
-
 // w <- fl32(w - eta_l g) (Sec. 3.2, Sec. 4.1); c <- RNE cast of the new w for FP16 / BF16 layers (Sec. 2).
 // One batch of the update.  `decision(seg, eta, code)` supplies the layer's step size and precision code.
 // MOM: the launch has a momentum buffer; its rows are loaded together with the weights and gradients, and fewer rows
 // are kept in flight.
-template <bool BF16, bool MOM, typename Decision>
+// STREAM_W: the new weights are stored with the streaming hint (first to leave L2), for callers that keep other data
+// in L2 on purpose.
+// ROWS: rows of loads a lane keeps in flight (0: the default for the gradient type).
+template <bool BF16, bool MOM, bool STREAM_W, int ROWS = 0, typename Decision>
 __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, const Decision &decision)
 {
-    constexpr int U = MOM ? (BF16 ? TA_APPLY_ROWS_BF16 : TA_APPLY_ROWS) / 2 : (BF16 ? TA_APPLY_ROWS_BF16 : TA_APPLY_ROWS);
+    constexpr int U0 = ROWS > 0 ? ROWS : (BF16 ? TA_APPLY_ROWS_BF16 : TA_APPLY_ROWS);
+    constexpr int U = MOM ? U0 / 2 : U0;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     {
         const uint32_t it = batch * kWarps + warp;
@@ -771,25 +856,7 @@ __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, 
                 gv.w = sgd_direction(gv.w, wv.w, A.mom ? &mv.w : nullptr, A.momentum, A.weight_decay);
                 if (A.mom) *reinterpret_cast<float4 *>(A.mom + i0) = mv;
             }
-            wv.x = fmaf(neg_eta, gv.x, wv.x);
-            wv.y = fmaf(neg_eta, gv.y, wv.y);
-            wv.z = fmaf(neg_eta, gv.z, wv.z);
-            wv.w = fmaf(neg_eta, gv.w, wv.w);
-            if (TA_APPLY_STREAM_W_STORE) __stcs(reinterpret_cast<float4 *>(A.w + i0), wv);
-            else *reinterpret_cast<float4 *>(A.w + i0) = wv;
-            if (code == 0u) {
-                const __half2 a = __floats2half2_rn(wv.x, wv.y), b = __floats2half2_rn(wv.z, wv.w);
-                uint2 o;
-                o.x = *reinterpret_cast<const uint32_t *>(&a);
-                o.y = *reinterpret_cast<const uint32_t *>(&b);
-                __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
-            } else if (code == 1u) {
-                const __nv_bfloat162 a = __floats2bfloat162_rn(wv.x, wv.y), b = __floats2bfloat162_rn(wv.z, wv.w);
-                uint2 o;
-                o.x = *reinterpret_cast<const uint32_t *>(&a);
-                o.y = *reinterpret_cast<const uint32_t *>(&b);
-                __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
-            }
+            update_store4<STREAM_W>(A.w, A.c, i0, wv, gv, neg_eta, code);
         };
 
         const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
@@ -830,7 +897,7 @@ __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
     if (A.status->skipped) return;
     const LayerState *state = A.state;
     auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) apply_batch<BF16, MOM>(A, batch, decision);
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) apply_batch<BF16, MOM, TA_APPLY_STREAM_W_STORE != 0>(A, batch, decision);
 }
 
 // ------------------------------------------------------------------ one launch for small models
@@ -856,9 +923,11 @@ __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
 
 // Statistics of one run, and of all runs of one layer inside one block.
 struct FusedPartial {
-    double s1, s2;               // sum and sum of squares of the gradient
+    double s1, s2;               // sums of (g - pivot) and (g - pivot)^2
     uint32_t amax, amin;         // largest / smallest |S| as bit patterns
-    uint32_t bad, pad;           // non-finite inputs
+    uint32_t bad;                // non-finite inputs
+    float pivot;                 // the first gradient value of the run (of the block's first run of the layer)
+    uint32_t n, pad;             // gradient values summed
 };
 
 // One slot: row `row` of the flat buffer, of which elements [lo, hi) (0..128 inside the row, packed as
@@ -1009,7 +1078,7 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
     float *sh_eta = reinterpret_cast<float *>(ptr);
     uint32_t *sh_code = reinterpret_cast<uint32_t *>(sh_eta + A.max_block_layers);
     static_assert(sizeof(LayerState) % 8 == 0, "LayerState is copied as 64-bit words");
-    static_assert(sizeof(FusedSlot) == 16 && sizeof(FusedPartial) == 32, "shared-memory layout");
+    static_assert(sizeof(FusedSlot) == 16 && sizeof(FusedPartial) == 40, "shared-memory layout");
     static_assert(sizeof(FusedWarpHead) == 16 && sizeof(FusedBlockHead) == 32 && sizeof(FusedBlockLayer) == 32, "plan records");
     constexpr uint32_t kStateWords = sizeof(LayerState) / 8;
 
@@ -1047,7 +1116,8 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
         SweepAcc<P, false> acc;
         uint32_t X[PP][4];
         uint64_t have_block = ~0ull;
-        uint32_t cur_run = 0u;
+        uint32_t cur_run = 0xFFFFFFFFu, run_n = 0u;
+        float run_pivot = 0.f;
         bool bad_seen = false;
         auto flush = [&](uint32_t run) {
             const double s1 = warp_sum(acc.s1), s2 = warp_sum(acc.s2);
@@ -1067,8 +1137,9 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
                 bad = __reduce_add_sync(0xFFFFFFFFu, bad);
                 bad_seen = bad_seen || bad != 0u;
             }
-            if (lane == 0) sh_run[run_lo - brun_lo + run] = FusedPartial{s1, s2, amax, amin, bad, 0u};
+            if (lane == 0) sh_run[run_lo - brun_lo + run] = FusedPartial{s1, s2, amax, amin, bad, run_pivot, run_n, 0u};
             acc = SweepAcc<P, false>();
+            run_n = 0u;
         };
         auto start_weight_copies = [&]() {
             const uint32_t n = min(n_slots, A.cap_w);
@@ -1105,7 +1176,17 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
             for (int u = 0; u < U; ++u) {
                 if (s0 + u < n_slots) {
                     const FusedSlot sl = sh_slot[s0 + u];
-                    if (sl.run != cur_run) { flush(cur_run); cur_run = sl.run; }
+                    const float gv[4] = {rd[u].g.x, rd[u].g.y, rd[u].g.z, rd[u].g.w};
+                    if (sl.run != cur_run) {
+                        // a new run: its first gradient value, held by one lane of this row, becomes the pivot of its sums
+                        if (cur_run != 0xFFFFFFFFu) flush(cur_run);
+                        cur_run = sl.run;
+                        const uint32_t first = sl.lo_hi & 0xFFFFu, comp = first & 3u;
+                        const float mine = comp == 0u ? gv[0] : (comp == 1u ? gv[1] : (comp == 2u ? gv[2] : gv[3]));
+                        run_pivot = __shfl_sync(0xFFFFFFFFu, mine, first >> 2);
+                        acc.pivot = (double)run_pivot;
+                    }
+                    run_n += (sl.lo_hi >> 16) - (sl.lo_hi & 0xFFFFu);
                     uint32_t e_lo, e_hi;
                     lane_range(sl, e_lo, e_hi);
                     uint32_t sel[PP];
@@ -1120,7 +1201,6 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
                     }
 #pragma unroll
                     for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
-                    const float gv[4] = {rd[u].g.x, rd[u].g.y, rd[u].g.z, rd[u].g.w};
 #pragma unroll
                     for (uint32_t e = 0; e < 4; ++e) {
                         if (e >= e_lo && e < e_hi) {
@@ -1147,10 +1227,12 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
     __syncthreads();
     for (uint32_t q = tid; q < nl; q += kThreads) {
         const uint32_t lo = sh_bl[q].run_lo, hi = sh_bl[q].run_hi;
-        FusedPartial t{0.0, 0.0, 0u, 0xFFFFFFFFu, 0u, 0u};
+        FusedPartial t{0.0, 0.0, 0u, 0xFFFFFFFFu, 0u, sh_run[lo - brun_lo].pivot, 0u, 0u};
         for (uint32_t r = lo; r < hi; ++r) {
             const FusedPartial x = sh_run[r - brun_lo];
-            t.s1 += x.s1; t.s2 += x.s2;
+            const MomentSums m = rebase(x.s1, x.s2, (double)x.n, (double)x.pivot, (double)t.pivot);
+            t.s1 += m.s1; t.s2 += m.s2;
+            t.n += x.n;
             t.amax = max(t.amax, x.amax); t.amin = min(t.amin, x.amin);
             t.bad += x.bad;
         }
@@ -1167,17 +1249,17 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
     const bool skip = __ldcg(A.barrier + 1) == A.epoch;
 
     // decisions of the layers this block touches, from the block partials of each (Sec. 3.1 - 3.4)
-    auto decide = [&](uint32_t q, double s1, double s2, uint32_t amax, uint32_t amin) {
+    auto decide = [&](uint32_t q, double pivot, double s1, double s2, uint32_t amax, uint32_t amin) {
         LayerState old;
         unsigned long long *dst = reinterpret_cast<unsigned long long *>(&old);
 #pragma unroll
         for (uint32_t i = 0; i < kStateWords; ++i) dst[i] = sh_old[q * kStateWords + i];
         const double n = sh_bl[q].n;
-        const double mu = s1 / n;
-        double var = s2 / n - mu * mu;
+        const double shift = s1 / n;
+        double var = s2 / n - shift * shift;
         if (!(var > 0.0)) var = 0.0;
         LayerScratch sc;
-        sc.mean = mu; sc.var = var; sc.sum_abs = 0.0; sc.bad = 0ull; sc.amax = amax; sc.amin = amin;
+        sc.mean = pivot + shift; sc.var = var; sc.sum_abs = 0.0; sc.bad = 0ull; sc.amax = amax; sc.amin = amin;
         uint32_t near;
         const LayerState st = decide_layer(A.dp, old, sc, near);
         sh_eta[q] = st.eta;
@@ -1190,22 +1272,28 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
         if (hi - lo > kThreadCombine) continue;
         double s1 = 0.0, s2 = 0.0;
         uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+        const double pivot = (double)__ldcg(&A.part[lo].pivot);
         for (uint32_t i = lo; i < hi; ++i) {
-            s1 += __ldcg(&A.part[i].s1);
-            s2 += __ldcg(&A.part[i].s2);
+            const MomentSums m = rebase(__ldcg(&A.part[i].s1), __ldcg(&A.part[i].s2), (double)__ldcg(&A.part[i].n),
+                                        (double)__ldcg(&A.part[i].pivot), pivot);
+            s1 += m.s1;
+            s2 += m.s2;
             amax = max(amax, __ldcg(&A.part[i].amax));
             amin = min(amin, __ldcg(&A.part[i].amin));
         }
-        decide(q, s1, s2, amax, amin);
+        decide(q, pivot, s1, s2, amax, amin);
     }
     for (uint32_t q = warp; q < nl; q += kWarps) {      // layers spread over many blocks: one warp each
         const uint32_t lo = sh_bl[q].part_lo, hi = sh_bl[q].part_hi;
         if (hi - lo <= kThreadCombine) continue;
         double s1 = 0.0, s2 = 0.0;
         uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+        const double pivot = (double)__ldcg(&A.part[lo].pivot);
         for (uint32_t i = lo + lane; i < hi; i += 32) {
-            s1 += __ldcg(&A.part[i].s1);
-            s2 += __ldcg(&A.part[i].s2);
+            const MomentSums m = rebase(__ldcg(&A.part[i].s1), __ldcg(&A.part[i].s2), (double)__ldcg(&A.part[i].n),
+                                        (double)__ldcg(&A.part[i].pivot), pivot);
+            s1 += m.s1;
+            s2 += m.s2;
             amax = max(amax, __ldcg(&A.part[i].amax));
             amin = min(amin, __ldcg(&A.part[i].amin));
         }
@@ -1213,7 +1301,7 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
         s2 = warp_sum(s2);
         amax = __reduce_max_sync(0xFFFFFFFFu, amax);
         amin = __reduce_min_sync(0xFFFFFFFFu, amin);
-        if (lane == 0) decide(q, s1, s2, amax, amin);
+        if (lane == 0) decide(q, pivot, s1, s2, amax, amin);
     }
     cp_async_wait_all();
     if (blockIdx.x == 0 && tid == 0) {
@@ -1798,7 +1886,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_resolve(const ApplyArgs A, c
     const LayerState *state = A.state;
     // eta and code were fixed by k_decide; resolve blocks write other fields (threshold, mass) of the same records
     auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
-    for (uint32_t batch = blockIdx.x - n_layers; batch < A.n_batches; batch += gridDim.x - n_layers) apply_batch<BF16, MOM>(A, batch, decision);
+    for (uint32_t batch = blockIdx.x - n_layers; batch < A.n_batches; batch += gridDim.x - n_layers) apply_batch<BF16, MOM, TA_APPLY_STREAM_W_STORE != 0>(A, batch, decision);
 }
 
 }  // namespace ta

@@ -7,6 +7,7 @@
 
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdio>
 
 namespace {
@@ -55,14 +56,17 @@ constexpr uint32_t kTileElems = TA_STATIC_TILE_ELEMS;     // elements one warp r
 constexpr uint32_t kMaxTiles = TA_STATIC_MAX_TILES;
 constexpr uint32_t kMaxLayers = TA_STATIC_MAX_LAYERS;
 
-// One partial per tile: sum, sum of squares, count of non-finite values.
+// One partial per tile: sums of (x - pivot) and (x - pivot)^2 with the tile's first value as pivot (so that a
+// layer whose mean dwarfs its spread loses no digits), that pivot, and the count of non-finite values.
 struct StaticScratch {
     double s1[kMaxTiles];
     double s2[kMaxTiles];
+    float pivot[kMaxTiles];
     uint32_t bad[kMaxTiles];
 };
 
-// The scratch itself.  Every GPU that loads this library holds these bytes until the process exits.
+// The scratch itself.  A GPU holds these bytes from the moment the CUDA runtime loads this file's device code on
+// it (with the runtime's default lazy loading: at the first call on that device) until the process exits.
 // In host code the name below is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
 
@@ -75,7 +79,7 @@ struct StaticTable {
 };
 
 constexpr int kMaxDevices = 64;
-StaticScratch *g_scratch_addr[kMaxDevices] = {};          // device address of the array, per device
+std::atomic<StaticScratch *> g_scratch_addr[kMaxDevices];  // device address of the array, per device (looked up once)
 thread_local char g_error[256] = "";
 
 template <bool BF16>
@@ -97,9 +101,10 @@ __global__ void __launch_bounds__(kThreads) k_moments_static_tiles(const StaticT
         const uint64_t end = (cell + 1) * kTileElems < seg_e ? (cell + 1) * kTileElems : seg_e;
         double s1 = 0.0, s2 = 0.0;
         uint32_t bad = 0;
+        const float pivot = load1<BF16>(g, begin);
         auto one = [&](float v) {
             if ((__float_as_uint(v) & 0x7FFFFFFFu) >= kNonFiniteBits) ++bad;
-            const double x = (double)v;
+            const double x = (double)v - (double)pivot;
             s1 += x;
             s2 = fma(x, x, s2);
         };
@@ -118,7 +123,7 @@ __global__ void __launch_bounds__(kThreads) k_moments_static_tiles(const StaticT
         s1 = warp_sum(s1);
         s2 = warp_sum(s2);
         bad = __reduce_add_sync(0xFFFFFFFFu, bad);
-        if (lane == 0) { scr->s1[tile] = s1; scr->s2[tile] = s2; scr->bad[tile] = bad; }
+        if (lane == 0) { scr->s1[tile] = s1; scr->s2[tile] = s2; scr->pivot[tile] = pivot; scr->bad[tile] = bad; }
     }
 }
 
@@ -129,9 +134,18 @@ __global__ void __launch_bounds__(kThreads) k_moments_static_layers(const Static
     __shared__ double red[kWarps];
     const uint32_t l = blockIdx.x;
     double s1 = 0.0, s2 = 0.0, bad = 0.0;
+    // the tiles summed around their own pivots; move every tile's sums to the pivot of the layer's first tile:
+    // with d = p_tile - p_layer, sum (x - p_layer) = s1 + n d and sum (x - p_layer)^2 = s2 + d (2 s1 + n d)
+    const uint64_t seg_b = T.offset[l], seg_e = seg_b + T.length[l];
+    const double p_layer = (double)scr->pivot[T.tile_lo[l]];
     for (uint32_t t = T.tile_lo[l] + threadIdx.x; t < T.tile_lo[l + 1]; t += kThreads) {
-        s1 += scr->s1[t];
-        s2 += scr->s2[t];
+        const uint64_t cell = seg_b / kTileElems + (t - T.tile_lo[l]);
+        const uint64_t begin = cell * kTileElems > seg_b ? cell * kTileElems : seg_b;
+        const uint64_t end = (cell + 1) * kTileElems < seg_e ? (cell + 1) * kTileElems : seg_e;
+        const double n = (double)(end - begin), d = (double)scr->pivot[t] - p_layer;
+        const double a = scr->s1[t];
+        s1 += fma(n, d, a);
+        s2 += fma(d, fma(n, d, 2.0 * a), scr->s2[t]);
         bad += (double)scr->bad[t];
     }
     s1 = block_sum(s1, red);
@@ -139,10 +153,10 @@ __global__ void __launch_bounds__(kThreads) k_moments_static_layers(const Static
     bad = block_sum(bad, red);
     if (threadIdx.x == 0) {
         const double n = (double)T.length[l];
-        const double mu = s1 / n;
-        double var = s2 / n - mu * mu;
+        const double shift = s1 / n;
+        double var = s2 / n - shift * shift;
         if (!(var > 0.0)) var = 0.0;
-        mean_var[2 * l] = mu;
+        mean_var[2 * l] = p_layer + shift;
         mean_var[2 * l + 1] = var;
         if (nonfinite) nonfinite[l] = (uint32_t)(bad > 4294967295.0 ? 4294967295.0 : bad);
     }
@@ -168,8 +182,9 @@ int ta_grad_moments_static(const ta_segment *table, uint32_t L, const void *g, u
     if (!table || !g || !mean_var || L == 0) return fail(TA_ERR_ARG, "ta_grad_moments_static: NULL argument or empty table");
     if (L > kMaxLayers) return fail(TA_ERR_ARG, "ta_grad_moments_static: more than TA_STATIC_MAX_LAYERS layers");
     if (grad_dtype != TA_GRAD_F32 && grad_dtype != TA_GRAD_BF16) return fail(TA_ERR_ARG, "ta_grad_moments_static: unknown grad_dtype");
-    if ((reinterpret_cast<uintptr_t>(g) & 15u) || (reinterpret_cast<uintptr_t>(mean_var) & 7u))
-        return fail(TA_ERR_ALIGN, "ta_grad_moments_static: g must be 16-byte aligned, mean_var 8-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(g) & 15u) || (reinterpret_cast<uintptr_t>(mean_var) & 7u) ||
+        (reinterpret_cast<uintptr_t>(nonfinite) & 3u))
+        return fail(TA_ERR_ALIGN, "ta_grad_moments_static: g must be 16-byte aligned, mean_var 8-byte, nonfinite 4-byte aligned");
     StaticTable T;
     uint64_t end = 0, tiles = 0;
     for (uint32_t l = 0; l < L; ++l) {
@@ -190,17 +205,20 @@ int ta_grad_moments_static(const ta_segment *table, uint32_t L, const void *g, u
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
         return fail(TA_ERR_CUDA, "ta_grad_moments_static: no current CUDA device");
-    if (!g_scratch_addr[dev]) {
-        // first call on this device: ask the runtime where this device's copy of the array lives
+    StaticScratch *scr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!scr) {
+        // first call on this device: ask the runtime where this device's copy of the array lives (this is also the
+        // moment the runtime loads this file's device code onto the device).  Threads that race here all get the
+        // same answer, so whichever store lands last changes nothing.
         void *p = nullptr;
         const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess || !p) {
             snprintf(g_error, sizeof(g_error), "ta_grad_moments_static: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
             return TA_ERR_CUDA;
         }
-        g_scratch_addr[dev] = static_cast<StaticScratch *>(p);
+        scr = static_cast<StaticScratch *>(p);
+        g_scratch_addr[dev].store(scr, std::memory_order_release);
     }
-    StaticScratch *scr = g_scratch_addr[dev];
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;

@@ -3,6 +3,7 @@
 #include "../../include/triaccel.h"
 
 #include <algorithm>
+#include <deque>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -10,6 +11,7 @@
 #include <vector>
 
 #include "kernels.cuh"
+#include "pipeline.cuh"
 
 namespace {
 
@@ -29,12 +31,19 @@ struct DeviceBuffers {
     ta::FusedSlot *slot_table = nullptr;
     ta::FusedPartial *part = nullptr;             // fused launch: block partials, grouped by layer
     double *p_s1 = nullptr, *p_s2 = nullptr, *p_sa = nullptr, *p_mass = nullptr;
+    float *p_piv = nullptr;
     uint32_t *p_amax = nullptr, *p_amin = nullptr, *p_bad = nullptr;
     float *abs_s = nullptr;
     uint32_t *hist = nullptr;
     ta::SelectState *sel = nullptr;
     uint32_t *mask = nullptr;
     uint32_t *cand_count = nullptr, *cand_val = nullptr, *cand_idx = nullptr, *batch_seg = nullptr;
+    // layer-pipelined pass (TA_FLAG_INPUTS_FINITE): its own items, task queues and counters
+    ta::PipeTask *pipe_tasks_sweep = nullptr, *pipe_tasks_apply = nullptr, *pipe_tasks_hold = nullptr;
+    uint32_t *pipe_batch_lo = nullptr;
+    ta::BatchSums *pipe_bsum = nullptr;
+    uint32_t *pipe_layer_done = nullptr, *pipe_layer_ready = nullptr;
+    ta::PipeControl *pipe_ctl = nullptr;
     // power iteration support: per-item partial sums, per-layer coefficients and norms
     double *pw_part = nullptr;
     float *pw_coef = nullptr, *pw_norm = nullptr;
@@ -72,6 +81,11 @@ struct ta_handle {
     size_t fused_smem = 0;
     unsigned long long barrier_base = 0;  // barrier arrivals of all fused launches so far
     unsigned long long fused_launches = 0;// fused launches since the arrival counters were last cleared
+    bool pipe_ok = false;                 // large dense models with TA_FLAG_INPUTS_FINITE: the layer-pipelined launch
+    uint32_t pipe_batches = 0;
+    int pipe_per_sm = 0;
+    unsigned long long pipe_base_s = 0, pipe_base_a = 0;
+    uint32_t pipe_launches = 0;
     std::vector<ta::Item> items_host;     // the plan, kept for the pipelined host path
     cudaStream_t copy_back = nullptr;     // ta_step_host: device-to-host copies run beside the host-to-device ones
     std::vector<cudaEvent_t> chunk_done;
@@ -106,7 +120,8 @@ template <typename T> cudaError_t dev_alloc(T **p, size_t count)
 
 void free_all(DeviceBuffers &d)
 {
-    void *ptrs[] = {d.warp_head, d.block_head, d.block_layer, d.slot_table, d.part, d.mom, d.pw_part, d.pw_coef, d.pw_norm, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2,
+    void *ptrs[] = {d.pipe_tasks_sweep, d.pipe_tasks_apply, d.pipe_tasks_hold, d.pipe_batch_lo, d.pipe_bsum, d.pipe_layer_done, d.pipe_layer_ready, d.pipe_ctl,
+                    d.warp_head, d.block_head, d.block_layer, d.slot_table, d.part, d.mom, d.pw_part, d.pw_coef, d.pw_norm, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2, d.p_piv,
                     d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
     for (void *p : ptrs)
@@ -118,10 +133,6 @@ void free_all(DeviceBuffers &d)
 // items, so that thousands of tiny tensors and a few huge ones both keep all SMs busy.
 uint32_t choose_item_elems(uint64_t n_params, int sm_count)
 {
-    if (const char *env = getenv("TRIACCEL_ITEM_ELEMS")) {
-        const long v = atol(env);
-        if (v >= 128 && v <= (1 << 20) && v % 128 == 0) return (uint32_t)v;
-    }
     const uint64_t want_items = (uint64_t)sm_count * ta::kWarps * 4;
     uint32_t best = 512;
     for (uint32_t cand : {1024u, 2048u, 4096u, 8192u, 16384u})
@@ -131,12 +142,7 @@ uint32_t choose_item_elems(uint64_t n_params, int sm_count)
 
 int grid_for(const ta_handle *h)
 {
-    int per_sm = 8;
-    if (const char *env = getenv("TRIACCEL_CTAS_PER_SM")) {
-        const int v = atoi(env);
-        if (v >= 1 && v <= 32) per_sm = v;
-    }
-    const long long cap = (long long)h->sm_count * per_sm;
+    const long long cap = (long long)h->sm_count * 8;
     return (int)std::max<long long>(1, std::min<long long>(h->n_batches, cap));
 }
 
@@ -313,11 +319,64 @@ RunPlan plan_runs(const ta_segment *table, uint32_t L, uint64_t max_warps)
     return pl;
 }
 
-uint64_t fused_max_params()
+// The plan of the layer-pipelined pass: batches of kPipeCells cells of kPipeItemElems elements cut on a global grid,
+// every batch inside one layer, and the task queues.  A step with decisions: the sweep tasks in buffer order, and the
+// apply tasks layer by layer, within a layer the last batch first.  A step without decisions: one single-pass task
+// per batch, in buffer order.
+struct PipePlan {
+    std::vector<uint32_t> batch_lo;
+    std::vector<ta::PipeTask> sweep, apply, hold;
+};
+
+PipePlan plan_pipe(const ta_segment *table, uint32_t L)
 {
-    if (const char *env = getenv("TRIACCEL_FUSED_MAX_PARAMS")) return (uint64_t)atoll(env);
-    return 16ull << 20;      // models up to ~16 M parameters (ResNet-18 scale) take the one-launch path
+    PipePlan pl;
+    pl.batch_lo.resize(L + 1);
+    std::vector<ta::PipeTask> batches;         // in buffer order; the kind is filled in per queue
+    const uint64_t cells = ta::kPipeCells;     // cells of kPipeItemElems elements per batch
+    for (uint32_t l = 0; l < L; ++l) {
+        pl.batch_lo[l] = (uint32_t)batches.size();
+        const uint64_t b = table[l].offset, e = b + table[l].length;
+        for (uint64_t p = b; p < e;) {
+            const uint64_t next = std::min<uint64_t>(e, (p / ta::kPipeItemElems + cells) * (uint64_t)ta::kPipeItemElems);
+            batches.push_back(ta::PipeTask{p, (uint32_t)(next - p), l, (uint32_t)batches.size(), 0u, 0u, 0u});
+            p = next;
+        }
+        for (uint32_t i = pl.batch_lo[l]; i < batches.size(); ++i) batches[i].layer_batches = (uint32_t)batches.size() - pl.batch_lo[l];
+    }
+    pl.batch_lo[L] = (uint32_t)batches.size();
+    auto task_of = [&](uint32_t b, uint32_t kind) {
+        ta::PipeTask t = batches[b];
+        t.seg_type |= kind << 30;
+        return t;
+    };
+    pl.hold.reserve(batches.size());
+    pl.sweep.reserve(batches.size());
+    pl.apply.reserve(batches.size());
+    for (uint32_t b = 0; b < batches.size(); ++b) {
+        pl.hold.push_back(task_of(b, ta::kTaskBoth));
+        pl.sweep.push_back(task_of(b, ta::kTaskSweep));
+    }
+    for (uint32_t l = 0; l < L; ++l)
+        for (uint32_t b = pl.batch_lo[l + 1]; b-- > pl.batch_lo[l];) pl.apply.push_back(task_of(b, ta::kTaskApply));
+    return pl;
 }
+
+template <int P, bool BF16> const void *pipe_fn() { return reinterpret_cast<const void *>(&ta::k_pipe<P, BF16>); }
+
+const void *pipe_kernel(int P, bool bf16)
+{
+    switch (P) {
+    case 0: return bf16 ? pipe_fn<0, true>() : pipe_fn<0, false>();
+    case 1: return bf16 ? pipe_fn<1, true>() : pipe_fn<1, false>();
+    case 2: return bf16 ? pipe_fn<2, true>() : pipe_fn<2, false>();
+    case 4: return bf16 ? pipe_fn<4, true>() : pipe_fn<4, false>();
+    case 8: return bf16 ? pipe_fn<8, true>() : pipe_fn<8, false>();
+    default: return nullptr;
+    }
+}
+
+constexpr uint64_t kFusedMaxParams = 16ull << 20;      // models up to ~16 M parameters (ResNet-18 scale) take the one-launch path
 
 // A bounded wait inside a kernel ran out (a block of a cooperative launch never arrived): the step that
 // hit it is incomplete.  Reports it once and re-arms the barrier.
@@ -331,6 +390,13 @@ int check_device_error(ta_handle *h)
     if (h->d.barrier) TA_CUDA(h, cudaMemset(h->d.barrier, 0, 2 * sizeof(unsigned long long)));
     h->barrier_base = 0;
     h->fused_launches = 0;
+    if (h->pipe_ok) {
+        TA_CUDA(h, cudaMemset(h->d.pipe_ctl, 0, sizeof(ta::PipeControl)));
+        TA_CUDA(h, cudaMemset(h->d.pipe_layer_done, 0, h->L * sizeof(uint32_t)));
+        TA_CUDA(h, cudaMemset(h->d.pipe_layer_ready, 0, h->L * sizeof(uint32_t)));
+        h->pipe_base_s = h->pipe_base_a = 0;
+        h->pipe_launches = 0;
+    }
     return fail(h, TA_ERR_CUDA, "a bounded device-side wait ran out during the last step; its results are incomplete");
 }
 
@@ -373,7 +439,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     if (hp->grad_dtype != TA_GRAD_F32 && hp->grad_dtype != TA_GRAD_BF16) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown grad_dtype");
     if (!(hp->momentum >= 0.f && hp->momentum < 1.f)) return fail(nullptr, TA_ERR_ARG, "ta_create: momentum must be in [0,1)");
     if (!(hp->weight_decay >= 0.f) || !(hp->weight_decay < 1e30f)) return fail(nullptr, TA_ERR_ARG, "ta_create: weight_decay must be finite and >= 0");
-    if (hp->flags != 0u) return fail(nullptr, TA_ERR_ARG, "ta_create: flags must be 0");
+    if (hp->flags & ~(uint32_t)(TA_FLAG_INPUTS_FINITE | TA_FLAG_NO_ONE_LAUNCH)) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown bit in flags");
     if (n_total % 4 != 0) return fail(nullptr, TA_ERR_ARG, "ta_create: n_total must be a multiple of 4");
     uint64_t end = 0, n_params = 0;
     for (uint32_t l = 0; l < L; ++l) {
@@ -422,7 +488,8 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     {
         int coop = 0;
         TA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device));
-        if (coop && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f && n_params <= fused_max_params()) {
+        if (coop && !(hp->flags & TA_FLAG_NO_ONE_LAUNCH) && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f &&
+            n_params <= kFusedMaxParams) {
             const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
             h->fused_ok = true;
             fused_per_sm = 1 << 20;
@@ -432,7 +499,6 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
                 TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(P, bf16), ta::kThreads, 0));
                 fused_per_sm = std::min(fused_per_sm, per_sm);
             }
-            if (const char *env = getenv("TRIACCEL_FUSED_CTAS_PER_SM")) fused_per_sm = std::min(fused_per_sm, std::max(1, atoi(env)));
             if (fused_per_sm < 1) h->fused_ok = false;
         }
     }
@@ -466,8 +532,6 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
             h->fused_cap_w = (uint32_t)std::min<long long>(pl.max_slots, rows_fit);
             h->fused_cap_g = (uint32_t)std::min<long long>(pl.max_slots, rows_fit - h->fused_cap_w);
             if (h->fused_cap_w < pl.max_slots) h->fused_cap_w = h->fused_cap_g = 0;
-            if (const char *env = getenv("TRIACCEL_FUSED_CAP_W")) h->fused_cap_w = std::min<uint32_t>(h->fused_cap_w, (uint32_t)atoi(env));
-            if (const char *env = getenv("TRIACCEL_FUSED_CAP_G")) h->fused_cap_g = std::min<uint32_t>(h->fused_cap_g, (uint32_t)atoi(env));
             h->fused_block_layers = pl.max_block_layers;
             h->fused_block_runs = pl.max_block_runs;
             h->fused_slots = pl.max_slots;
@@ -522,6 +586,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     TA_TRY(dev_alloc(&d.status, 1));
     TA_TRY(dev_alloc(&d.p_s1, h->n_items));
     TA_TRY(dev_alloc(&d.p_s2, h->n_items));
+    TA_TRY(dev_alloc(&d.p_piv, h->n_items));
     TA_TRY(dev_alloc(&d.p_amax, h->n_items));
     TA_TRY(dev_alloc(&d.p_amin, h->n_items));
     TA_TRY(dev_alloc(&d.p_bad, h->n_items));
@@ -583,6 +648,40 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
             if ((long long)per_sm * h->sm_count < h->fused_grid) {
                 snprintf(h->err, 256, "ta_create: the one-launch grid of %d blocks is not resident (%d per SM)", h->fused_grid, per_sm);
                 return bail(TA_ERR_CUDA);
+            }
+        }
+    }
+    if ((hp->flags & TA_FLAG_INPUTS_FINITE) && !h->fused_ok && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f) {
+        // the layer-pipelined launch: its own (finer) items, the two task queues and the per-layer counters
+        const PipePlan pl = plan_pipe(table, L);
+        if (L < (1u << 30) && pl.sweep.size() < 0xFFFFFFFFull) {
+            const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
+            int per_sm = 1 << 20;
+            for (int P : {0, (int)hp->num_probes}) {
+                int v = 0;
+                TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, pipe_kernel(P, bf16), ta::kThreads, 0));
+                per_sm = std::min(per_sm, v);
+            }
+            if (per_sm >= 1) {
+                h->pipe_ok = true;
+                h->pipe_per_sm = per_sm;
+                h->pipe_batches = pl.batch_lo[L];
+                const size_t bytes = pl.sweep.size() * sizeof(ta::PipeTask);
+                TA_TRY(dev_alloc(&d.pipe_tasks_sweep, pl.sweep.size()));
+                TA_TRY(cudaMemcpy(d.pipe_tasks_sweep, pl.sweep.data(), bytes, cudaMemcpyHostToDevice));
+                TA_TRY(dev_alloc(&d.pipe_tasks_apply, pl.apply.size()));
+                TA_TRY(cudaMemcpy(d.pipe_tasks_apply, pl.apply.data(), bytes, cudaMemcpyHostToDevice));
+                TA_TRY(dev_alloc(&d.pipe_tasks_hold, pl.hold.size()));
+                TA_TRY(cudaMemcpy(d.pipe_tasks_hold, pl.hold.data(), bytes, cudaMemcpyHostToDevice));
+                TA_TRY(dev_alloc(&d.pipe_batch_lo, L + 1));
+                TA_TRY(cudaMemcpy(d.pipe_batch_lo, pl.batch_lo.data(), (L + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice));
+                TA_TRY(dev_alloc(&d.pipe_bsum, h->pipe_batches));
+                TA_TRY(dev_alloc(&d.pipe_layer_done, L));
+                TA_TRY(dev_alloc(&d.pipe_layer_ready, L));
+                TA_TRY(dev_alloc(&d.pipe_ctl, 1));
+                TA_TRY(cudaMemset(d.pipe_layer_done, 0, L * sizeof(uint32_t)));
+                TA_TRY(cudaMemset(d.pipe_layer_ready, 0, L * sizeof(uint32_t)));
+                TA_TRY(cudaMemset(d.pipe_ctl, 0, sizeof(ta::PipeControl)));
             }
         }
     }
@@ -658,6 +757,26 @@ int ta_plan_one_launch(const ta_segment *table, uint32_t L, uint32_t warps, ta_r
     return TA_OK;
 }
 
+int ta_plan_pipeline(const ta_segment *table, uint32_t L, uint32_t with_decisions, ta_task *out, uint64_t cap, uint64_t *n_tasks)
+{
+    if (!table || L == 0 || !n_tasks) return fail(nullptr, TA_ERR_ARG, "ta_plan_pipeline: table, L and n_tasks are required");
+    uint64_t end = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        if (table[l].length == 0 || table[l].length > 0xFFFFFFFEull)
+            return fail(nullptr, TA_ERR_ARG, "ta_plan_pipeline: segment length out of range");
+        if (table[l].offset < end) return fail(nullptr, TA_ERR_ARG, "ta_plan_pipeline: segments must be ascending and non-overlapping");
+        end = table[l].offset + table[l].length;
+    }
+    const PipePlan pl = plan_pipe(table, L);
+    std::vector<ta::PipeTask> tasks = with_decisions ? pl.sweep : pl.hold;
+    if (with_decisions) tasks.insert(tasks.end(), pl.apply.begin(), pl.apply.end());
+    *n_tasks = tasks.size();
+    if (tasks.size() > cap || (!out && cap)) return fail(nullptr, TA_ERR_ARG, "ta_plan_pipeline: out is too small for the queues");
+    for (size_t i = 0; i < tasks.size() && out; ++i)
+        out[i] = ta_task{tasks[i].begin, tasks[i].len, tasks[i].seg_type & 0x3FFFFFFFu, tasks[i].seg_type >> 30, 0u};
+    return TA_OK;
+}
+
 int ta_timing_begin(ta_handle *h, uint32_t max_steps)
 {
     if (!h) return TA_ERR_ARG;
@@ -711,6 +830,35 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
     cudaEvent_t *ev = timed ? &h->events[4 * (size_t)h->timed_used] : nullptr;
     if (timed) cudaEventRecord(ev[0], s);
 
+    if (h->pipe_ok && !defer_apply) {
+        const bool control = (step % h->hp.t_ctrl) == 0;
+        ta::PipeArgs pa{};
+        pa.tasks_s = control ? d.pipe_tasks_sweep : d.pipe_tasks_hold;
+        pa.tasks_a = d.pipe_tasks_apply;
+        pa.n_s = h->pipe_batches;
+        pa.n_a = control ? h->pipe_batches : 0u;
+        pa.batch_lo = d.pipe_batch_lo; pa.seg_len = d.seg_len; pa.bsum = d.pipe_bsum;
+        pa.layer_done = d.pipe_layer_done; pa.layer_ready = d.pipe_layer_ready; pa.ctl = d.pipe_ctl;
+        pa.base_s = h->pipe_base_s; pa.base_a = h->pipe_base_a; pa.epoch = h->pipe_launches + 1;
+        pa.w = w; pa.g = g; pa.hz = Hz; pa.c = c; pa.n_total = h->n_total; pa.seed = probe_seed; pa.step32 = (uint32_t)step;
+        pa.state = d.state; pa.scratch = d.scratch; pa.status = d.status;
+        pa.dp.hp = hyper_of(h->hp); pa.dp.eta0 = h->hp.eta0; pa.dp.has_hz = Hz ? 1u : 0u;
+        pa.dp.control = control ? 1u : 0u; pa.dp.topk = 0u;
+        pa.L = h->L; pa.step = step;
+        const unsigned grid = (unsigned)std::min<long long>((long long)h->sm_count * h->pipe_per_sm, pa.n_s);
+        void *args[] = {&pa};
+        TA_CUDA(h, cudaLaunchKernel(pipe_kernel(P, bf16), dim3(grid), dim3(ta::kThreads), args, 0, s));
+        h->pipe_base_s += (unsigned long long)pa.n_s + grid;     // every block draws exactly one ticket past the end of each queue
+        h->pipe_base_a += (unsigned long long)pa.n_a + grid;
+        ++h->pipe_launches;
+        ++h->launches;
+        if (timed) { cudaEventRecord(ev[1], s); cudaEventRecord(ev[2], s); cudaEventRecord(ev[3], s); ++h->timed_used; }
+        h->stepped = true;
+        h->last_step = step;
+        h->last_stream = s;
+        return TA_OK;
+    }
+
     if (h->fused_ok) {
         ta::FusedArgs fa{};
         fa.runs = d.items; fa.n_runs = h->n_items;
@@ -725,9 +873,7 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
         fa.max_slots = h->fused_slots; fa.max_block_runs = h->fused_block_runs; fa.max_block_layers = h->fused_block_layers;
         fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base;
         fa.epoch = h->fused_launches + 1;
-        // the weight copies start after the sweep (measured faster than starting them with its first loads)
-        static const bool early_w = getenv("TRIACCEL_FUSED_EARLY_W") ? atoi(getenv("TRIACCEL_FUSED_EARLY_W")) != 0 : false;
-        fa.early_weights = early_w ? 1u : 0u;
+        fa.early_weights = 0u;      // the weight copies start after the sweep (measured faster than starting them with its first loads)
         if (h->expire_next_wait) { fa.barrier_base += 1ull << 40; h->expire_next_wait = false; }
         const int grid = h->fused_grid;
         void *args[] = {&fa};
@@ -745,7 +891,7 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
     ta::SweepArgs sa{};
     sa.items = d.items; sa.n_items = h->n_items; sa.n_batches = h->n_batches;
     sa.g = g; sa.hz = Hz; sa.n_total = h->n_total; sa.seed = probe_seed; sa.step = (uint32_t)step;
-    sa.p_s1 = d.p_s1; sa.p_s2 = d.p_s2; sa.p_sa = d.p_sa;
+    sa.p_s1 = d.p_s1; sa.p_s2 = d.p_s2; sa.p_sa = d.p_sa; sa.p_piv = d.p_piv;
     sa.p_amax = d.p_amax; sa.p_amin = d.p_amin; sa.p_bad = d.p_bad;
     sa.abs_s = d.abs_s; sa.hist = d.hist; sa.batch_seg = d.batch_seg;
     const bool ok = bf16 ? dispatch_sweep<true>(h, P, sa, s) : dispatch_sweep<false>(h, P, sa, s);
@@ -753,8 +899,8 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
     if (timed) cudaEventRecord(ev[1], s);
 
     ta::DecideArgs da{};
-    da.item_lo = d.item_lo; da.seg_len = d.seg_len;
-    da.p_s1 = d.p_s1; da.p_s2 = d.p_s2; da.p_sa = d.p_sa;
+    da.item_lo = d.item_lo; da.seg_len = d.seg_len; da.items = d.items;
+    da.p_s1 = d.p_s1; da.p_s2 = d.p_s2; da.p_sa = d.p_sa; da.p_piv = d.p_piv;
     da.p_amax = d.p_amax; da.p_amin = d.p_amin; da.p_bad = d.p_bad;
     da.scratch = d.scratch; da.state = d.state; da.status = d.status;
     da.hp = hyper_of(h->hp); da.eta0 = h->hp.eta0; da.L = h->L;

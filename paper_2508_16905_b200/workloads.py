@@ -149,6 +149,9 @@ def get(name, **overrides):
     elif name == "gpt_1block":
         # one decoder block plus the embedding: the 1.3B workload's tensor mix at a size a profiler can replay
         w = dict(shapes=gpt_shapes(layers=1), steps=20, grad_dtype="bf16", d_low=1e-6)
+    elif name == "gpt_3block":
+        # three decoder blocks behind a small embedding: layers of the 1.3B workload's sizes, no tensor beyond L2
+        w = dict(shapes=gpt_shapes(layers=3, vocab=8192), steps=20, grad_dtype="bf16", d_low=1e-6)
     else:
         raise KeyError(name)
     w.update(overrides)

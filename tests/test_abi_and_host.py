@@ -6,6 +6,7 @@ import re
 import subprocess
 import sys
 
+import numpy as np
 import pytest
 import torch
 
@@ -51,7 +52,7 @@ def test_create_rejects_bad_arguments_before_touching_a_device():
         dict(table=[(0, 8)], n_total=8, t_ctrl=0),
         dict(table=[(0, 8)], n_total=8, momentum=1.0),
         dict(table=[(0, 8)], n_total=8, weight_decay=-1.0),
-        dict(table=[(0, 8)], n_total=8, flags=1),
+        dict(table=[(0, 8)], n_total=8, flags=4),                # unknown flag bit
         dict(table=[(0, 8)], n_total=8, tau_low=2.0, tau_high=1.0),
     ]
     for kw in bad:
@@ -137,6 +138,36 @@ def test_generators_are_seeded_and_have_the_stated_distributions():
     g = W.make_grads(heavy, 1)
     assert float((g.abs() > 8e-3).float().mean()) > 1e-4          # the Student-t(2) tail is present
     assert W.make_grads(W.get("gpt_1p3b", shapes=W.gpt_shapes(layers=1, d=64, vocab=128)), 1).dtype == torch.bfloat16
+
+
+def test_pipeline_queues_cover_every_layer_once():
+    rng = np.random.default_rng(5)
+    tables = [W.get("gpt_1p3b").table, W.get("resnet18_cifar", align=1).table]
+    off, t = 3, []
+    for _ in range(60):
+        n = int(rng.choice([1, 7, 2048, 2049, 14336, 14337, 50000, 3000000]))
+        off += int(rng.integers(0, 9))
+        t.append((off, n))
+        off += n
+    tables.append(t)
+    for table in tables:
+        hold = ta.ta_plan_pipeline(table, False)
+        both = ta.ta_plan_pipeline(table, True)
+        assert all(k == 2 for k, _, _, _ in hold) and len(both) == 2 * len(hold)
+        # the batches tile every layer exactly, in buffer order, on a grid of 2048-element cells
+        pos = {l: off for l, (off, n) in enumerate(table)}
+        for _, l, b, n in hold:
+            assert b == pos[l] and 0 < n <= 14336 and (b + n == table[l][0] + table[l][1] or (b + n) % 2048 == 0)
+            pos[l] += n
+        assert all(pos[l] == off + n for l, (off, n) in enumerate(table))
+        sweeps, applies = both[:len(hold)], both[len(hold):]
+        assert all(k == 0 for k, _, _, _ in sweeps) and all(k == 1 for k, _, _, _ in applies)
+        assert [x[1:] for x in sweeps] == [x[1:] for x in hold]
+        # update tasks: layer by layer, a layer's last batch first
+        assert [l for _, l, _, _ in applies] == sorted(l for _, l, _, _ in applies)
+        for l in range(len(table)):
+            mine = [x[1:] for x in applies if x[1] == l]
+            assert mine == [x[1:] for x in sweeps if x[1] == l][::-1]
 
 
 def test_replica_bookkeeping_world_size_2_gloo(tmp_path):
