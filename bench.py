@@ -4,9 +4,11 @@
 
 Prints ONE JSON line.  `value` is parameters per second of the whole job (N replicas), inputs
 resident in HBM; `e2e` is the same metric through ta_step_host with pinned HOST buffers
-(copies inside the timed region); `roofline` describes the dominant kernel (the update + cast
-kernel) against the measured HBM copy rate; `cpu_baseline` is the CPU checker timed on a
-bounded sample of the same workload.  `--impl reference` times the CPU checker alone.
+(copies inside the timed region); `roofline` describes the dominant kernel against the measured HBM copy rate
+(and, under `step`, the whole step against that rate and the 8 TB/s nominal peak, with the targets);
+`configs` carries the same figures for all five configurations and `paths` those of the passes a caller
+can opt into; `cpu_baseline` is the CPU checker timed on a bounded sample of the same workload.
+`--impl reference` times the CPU checker alone.
 """
 import argparse
 import hashlib
@@ -37,24 +39,11 @@ def measured_peak():
 
 def kernel_source_hash():
     h = hashlib.sha256()
-    with open(os.path.join(ROOT, "paper_2508_16905_b200", "csrc", "kernels.cuh"), "rb") as f:
-        h.update(f.read())
+    csrc = os.path.join(ROOT, "paper_2508_16905_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(f.read())
     return h.hexdigest()[:16]
-
-
-def recorded_traffic(workload, units):
-    """(DRAM bytes per launch of the dominant kernel, DRAM bytes per step over all kernels) from the committed ncu
-    captures, or (None, None) when there is none for this workload or the kernel source changed since."""
-    try:
-        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
-            rec = json.load(f)
-        if rec.get("kernels_cuh_sha256_16") != kernel_source_hash():
-            return None, None
-        w = rec["workloads"][workload]
-        per_kernel = w["dram_bytes_per_param"]
-        return per_kernel[w["dominant"]] * units, sum(per_kernel.values()) * units
-    except Exception:
-        return None, None
 
 
 class ClockSampler:
@@ -197,26 +186,37 @@ def run_reference(args):
     return 0
 
 
-def run_ours(args):
+TARGETS = {"gpt_1p3b": 0.75, "efficientnet_b0_cifar": 0.50}     # whole-step algorithmic GB/s over the 8 TB/s nominal peak
+
+
+def algorithmic_bytes(wl, codes, momentum=False):
+    """What the method itself must move per step, by kernel: (sweep, update, whole step)."""
+    g_b = 2 if wl.grad_dtype == "bf16" else 4
+    P, n = wl.num_probes, wl.num_params
+    topk = wl.topk_ppm < 1000000
+    copy_params = sum(m for (_, m), cd in zip(wl.table, codes) if cd < 2)
+    mom_b = 8 if momentum else 0
+    sweep = n * (g_b + 4 * P) + (4 * n if topk else 0)                       # top-k: |S| is written for the selection
+    update_reads, update_writes = n * (4 + g_b + mom_b // 2), n * (4 + mom_b // 2) + 2 * copy_params
+    step = n * (4 + g_b + 4 * P + 4 + mom_b) + 2 * copy_params + (n / 8 if topk else 0)
+    return {"sweep": sweep, "update": update_reads + update_writes, "update_writes": update_writes, "step": step,
+            "step_writes": 4 * n + 2 * copy_params + (n / 8 if topk else 0) + (4 * n if momentum else 0)}
+
+
+def measure(wl, hp, steps, warmup, dev, props, sample_clocks):
+    """Times `steps` optimizer passes of workload `wl` (inputs resident in HBM, rotating buffer sets where one step's
+    data would fit in L2), then the same number once more with the library's per-phase events.  Returns a dict."""
     import torch
     import paper_2508_16905_b200 as ta
     from paper_2508_16905_b200 import dist as D
     from paper_2508_16905_b200 import workloads as W
 
-    rank, local_rank, world = D.init("nccl")
-    torch.cuda.set_device(local_rank if world > 1 else 0)
-    dev = torch.device("cuda", torch.cuda.current_device())
-    props = torch.cuda.get_device_properties(dev)
-    wl = W.get(args.config, **({"t_ctrl": args.t_ctrl} if args.t_ctrl else {}))
-    steps, warmup = max(1, args.steps), max(3, args.warmup)
     P, N = wl.num_probes, wl.n_total
     l2_bytes = props.L2_cache_size
-
     bytes_in_per_set = N * ((2 if wl.grad_dtype == "bf16" else 4) + 4 * P)
     state_bytes = N * 6
     # rotate over R buffer sets so that consecutive steps never find their inputs in L2
     R = 1 if (bytes_in_per_set + state_bytes) > 4 * l2_bytes else max(2, -(-6 * l2_bytes // (bytes_in_per_set + state_bytes)))
-    hp = dict(wl.hparams(), momentum=args.momentum, weight_decay=args.weight_decay, flags=1 if args.inputs_finite else 0)
     h = ta.ta_create(wl.table, N, **hp)
     curv = W.make_curvature(wl, dev)
     sets = []
@@ -242,7 +242,8 @@ def run_ours(args):
         one_step(t)
     torch.cuda.synchronize()
     D.barrier()
-    sampler = ClockSampler(str(props.uuid) if str(props.uuid).startswith("GPU-") else "GPU-" + str(props.uuid)) if rank == 0 else None
+    uuid = str(props.uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid) if sample_clocks else None
     launches0 = ta.ta_launch_count(h)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -263,10 +264,102 @@ def run_ours(args):
         one_step(t)
     ms_sweep, ms_decide, ms_update, n_timed = ta.ta_timing_end(h)
     clocks = sampler.stop() if sampler else None
-    ms, units = D.aggregate(ms_local, wl.num_params * steps, device=dev)
     stats, status = ta.ta_stats(h)
-    codes = [s.code for s in stats]
     assert status.skipped == 0, "a benchmark step was skipped (non-finite synthetic input?)"
+    n_timed = max(1, n_timed)
+    out = {"ms_local": ms_local, "launches": int(launches), "codes": [s.code for s in stats], "clocks": clocks, "R": R,
+           "bytes_in_per_set": bytes_in_per_set, "state_bytes": state_bytes, "l2_bytes": l2_bytes, "sets": sets,
+           "phases": {"sweep": ms_sweep / n_timed, "decide_select": ms_decide / n_timed, "update": ms_update / n_timed}}
+    ta.ta_destroy(h)
+    return out
+
+
+def recorded_reads(workload):
+    """DRAM bytes read per parameter by each kernel of this workload, from the committed ncu captures; None when there
+    is no capture or a kernel source changed since."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
+            rec = json.load(f)
+        if rec.get("sources_sha256_16") != kernel_source_hash():
+            return None
+        return rec["workloads"][workload]
+    except Exception:
+        return None
+
+
+def describe(wl, m, steps, ms, peak, peak_kind, momentum=False, pipelined=False):
+    """Throughput and roofline figures of one measured workload."""
+    ab = algorithmic_bytes(wl, m["codes"], momentum)
+    ms_step = ms / steps
+    one_launch = m["launches"] == steps                   # the whole step in one kernel (one-launch or pipelined path)
+    ph = m["phases"]
+    if one_launch:
+        name, k_bytes, k_writes, k_ms = "whole step in one launch", ab["step"], ab["step_writes"], ms_step
+    elif ph["sweep"] > ph["update"]:                      # e.g. four probes + top-k: the sweep is the longest kernel
+        name, k_bytes, k_writes, k_ms = "k_sweep (statistics + Hutchinson sums)", ab["sweep"], (4 * wl.num_params if wl.topk_ppm < 1000000 else 0), ph["sweep"]
+    else:
+        name, k_bytes, k_writes, k_ms = "k_apply (master update + cast)", ab["update"], ab["update_writes"], ph["update"]
+    achieved = k_bytes / (k_ms * 1e-3) / 1e9
+    step_gbs = ab["step"] / (ms_step * 1e-3) / 1e9
+    # measured DRAM traffic of the dominant kernel: its reads per parameter from an ncu capture of a workload small
+    # enough to replay, times this workload's parameters; its writes are taken as the algorithmic writes of this run's
+    # own code mix (lines still dirty in L2 at the end of a captured launch are a constant, not a share)
+    traffic = None
+    rec = recorded_reads(wl.name)
+    key = ("k_pipe" if pipelined else "k_fused") if one_launch else ("k_sweep" if ph["sweep"] > ph["update"] else "k_apply")
+    if rec and key in rec.get("dram_read_bytes_per_param", {}):
+        traffic = max(rec["dram_read_bytes_per_param"][key] * wl.num_params + k_writes, k_bytes)
+    codes = m["codes"]
+    R = m["R"]
+    per_set = (m["bytes_in_per_set"] + m["state_bytes"]) / 1e6
+    l2 = (f"inputs of one step ({per_set:.0f} MB) exceed L2 ({m['l2_bytes'] / 1e6:.0f} MB)" if R == 1 else
+          f"{R} rotating buffer sets ({R * per_set:.0f} MB) exceed L2 ({m['l2_bytes'] / 1e6:.0f} MB)")
+    roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": peak_kind, "traffic": traffic, "algorithmic_bytes_per_launch": k_bytes, "ms_per_launch": k_ms,
+                "phases_ms_per_step": None if one_launch else ph,
+                "sweep_achieved_gbs": None if one_launch else ab["sweep"] / (ph["sweep"] * 1e-3) / 1e9,
+                "step": {"algorithmic_bytes": ab["step"], "achieved_gbs": step_gbs, "frac_of_peak": step_gbs / peak,
+                         "frac_of_8tbs_nominal": step_gbs / 8000.0}}
+    if wl.name in TARGETS:
+        roofline["step"]["target_frac_of_8tbs_nominal"] = TARGETS[wl.name]
+        roofline["step"]["target_met"] = step_gbs / 8000.0 >= TARGETS[wl.name]
+    summary = {"ms_per_step": ms_step, "params_per_s": wl.num_params / (ms_step * 1e-3), "params": wl.num_params,
+               "layers": len(wl.table), "algorithmic_bytes": ab["step"], "hbm_gbs_algorithmic": step_gbs,
+               "frac_of_measured": step_gbs / peak, "frac_of_8tbs_nominal": step_gbs / 8000.0,
+               "codes": {"fp16": codes.count(0), "bf16": codes.count(1), "fp32": codes.count(2)},
+               "launches_per_step": m["launches"] / steps, "l2": l2, "clocks": m["clocks"]}
+    if wl.name in TARGETS:
+        summary["target_frac_of_8tbs_nominal"] = TARGETS[wl.name]
+        summary["target_met"] = summary["frac_of_8tbs_nominal"] >= TARGETS[wl.name]
+    return roofline, summary, l2
+
+
+def run_ours(args):
+    import torch
+    import paper_2508_16905_b200 as ta
+    from paper_2508_16905_b200 import dist as D
+    from paper_2508_16905_b200 import workloads as W
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand for several GPUs: become one rank per GPU (one replica each)
+        os.execvp(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+                                   "--master-addr", "127.0.0.1", "--master-port", str(29500 + os.getpid() % 500),
+                                   os.path.abspath(__file__)] + sys.argv[1:])
+    rank, local_rank, world = D.init("nccl")
+    torch.cuda.set_device(local_rank if world > 1 else 0)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    props = torch.cuda.get_device_properties(dev)
+    over = {"t_ctrl": args.t_ctrl} if args.t_ctrl else {}
+    wl = W.get(args.config, **over)
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    P, N = wl.num_probes, wl.n_total
+    flags = ta.TA_FLAG_INPUTS_FINITE if args.inputs_finite else 0
+    hp = dict(wl.hparams(), momentum=args.momentum, weight_decay=args.weight_decay, flags=flags)
+    peak, peak_kind = measured_peak()
+
+    m = measure(wl, hp, steps, warmup, dev, props, sample_clocks=(rank == 0))
+    ms, units = D.aggregate(m["ms_local"], wl.num_params * steps, device=dev)
+    sets = m.pop("sets")
 
     # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
     e2e = None
@@ -289,62 +382,64 @@ def run_ours(args):
         span = wl.table[-1][0] + wl.table[-1][1] - wl.table[0][0]
         ms2, units2 = D.aggregate(dt_ms, wl.num_params * e2e_steps, device=dev)
         e2e = {"value": units2 / (ms2 / 1e3), "unit": UNIT, "steps": e2e_steps, "ms_per_step": ms2 / e2e_steps,
-               "h2d_bytes_per_step": int(bytes_in_per_set + 4 * N), "d2h_bytes_per_step": int(4 * span + 2 * copy_params),
+               "h2d_bytes_per_step": int(m["bytes_in_per_set"] + 4 * N), "d2h_bytes_per_step": int(4 * span + 2 * copy_params),
                "api": "ta_step_host (pinned host tensors in, new weights and 16-bit copies out)"}
         del wh, gh, hzh, ch
         ta.ta_destroy(h2)
+    del sets
+    torch.cuda.empty_cache()
+
+    # ---- one replica only: the other configurations, and the paths a caller can opt into
+    configs, paths = None, None
+    if world == 1 and not args.headline_only:
+        roofline0, summary0, _ = describe(wl, m, steps, ms, peak, peak_kind, bool(args.momentum))
+        configs = {wl.name: summary0}
+        for name in W.NAMES:
+            if name == wl.name:
+                continue
+            w2 = W.get(name)
+            k = max(steps, 50) if w2.num_params < 5e7 else steps
+            m2 = measure(w2, w2.hparams(), k, warmup, dev, props, sample_clocks=True)
+            m2.pop("sets")
+            torch.cuda.empty_cache()
+            configs[name] = describe(w2, m2, k, m2["ms_local"], peak, peak_kind)[1]
+        big_dense = wl.topk_ppm == 1000000 and wl.num_params > (16 << 20) and not args.momentum and not args.weight_decay
+        if big_dense and not args.inputs_finite:
+            # TA_FLAG_INPUTS_FINITE: the caller vouches for finite inputs; a step with decisions (this workload decides at
+            # every step) and a step between decisions (T_ctrl beyond the run: the single pass)
+            paths = {"flag": "TA_FLAG_INPUTS_FINITE"}
+            for label, extra in (("step_with_decisions", {}), ("step_between_decisions", {"t_ctrl": 1000000})):
+                w3 = W.get(args.config, **dict(over, **extra))
+                for which, fl in (("default", 0), ("inputs_finite", ta.TA_FLAG_INPUTS_FINITE)):
+                    if label == "step_with_decisions" and which == "default":
+                        paths.setdefault(label, {})[which] = summary0
+                        continue
+                    m3 = measure(w3, dict(w3.hparams(), flags=fl), steps, warmup, dev, props, sample_clocks=True)
+                    m3.pop("sets")
+                    torch.cuda.empty_cache()
+                    paths.setdefault(label, {})[which] = describe(w3, m3, steps, m3["ms_local"], peak, peak_kind, pipelined=bool(fl))[1]
 
     if rank != 0:
         D.shutdown()
         return 0
 
-    # ---- roofline of the dominant kernel (update + cast): algorithmic bytes / its measured duration
-    peak, peak_kind = measured_peak()
-    g_b = 2 if wl.grad_dtype == "bf16" else 4
-    copy_params = sum(n for (_, n), cd in zip(wl.table, codes) if cd < 2)
-    mom_b = 8 if args.momentum else 0          # momentum buffer read + write
-    update_bytes = wl.num_params * (4 + g_b + 4 + mom_b) + 2 * copy_params
-    sweep_bytes = wl.num_params * (g_b + 4 * P)
-    fused = int(launches) == steps          # small dense models run as one cooperative launch per step (k_fused)
-    step_bytes_min = wl.num_params * (4 + g_b + 4 * P + 4 + mom_b) + 2 * copy_params + (wl.num_params / 8 if wl.topk_ppm < 1000000 else 0)
-    ms_step = ms / steps
-    if fused:
-        update_bytes, upd_ms = step_bytes_min, ms_step        # one kernel per step: its duration is the step time
-    else:
-        upd_ms = ms_update / max(1, n_timed)
-    kernel_name = "k_fused (sweep + decisions + update in one launch)" if fused else "k_apply (master update + cast)"
-    if not fused and ms_sweep > ms_update:          # e.g. four probes + top-k: the sweep is the longest kernel
-        kernel_name, update_bytes, upd_ms = "k_sweep (statistics + Hutchinson sums)", sweep_bytes + (4 * wl.num_params if wl.topk_ppm < 1000000 else 0), ms_sweep / max(1, n_timed)
-    achieved = update_bytes / (upd_ms * 1e-3) / 1e9
-    traffic_kernel, traffic_step = recorded_traffic(wl.name, wl.num_params)
-    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-                "traffic": traffic_kernel,
-                "algorithmic_bytes_per_launch": update_bytes, "ms_per_launch": upd_ms,
-                "phases_ms_per_step": (None if fused else {"sweep": ms_sweep / max(1, n_timed), "decide_select": ms_decide / max(1, n_timed),
-                                                            "update": ms_update / max(1, n_timed)}),
-                "sweep_achieved_gbs": None if fused else sweep_bytes / (ms_sweep / max(1, n_timed) * 1e-3) / 1e9,
-                "step": {"algorithmic_bytes": step_bytes_min, "achieved_gbs": step_bytes_min / (ms_step * 1e-3) / 1e9,
-                         "frac_of_peak": step_bytes_min / (ms_step * 1e-3) / 1e9 / peak,
-                         "frac_of_8tbs_nominal": step_bytes_min / (ms_step * 1e-3) / 1e9 / 8000.0,
-                         "dram_bytes_measured": traffic_step,
-                         "dram_gbs_measured": (traffic_step / (ms_step * 1e-3) / 1e9) if traffic_step else None}}
-
+    roofline, summary, l2 = describe(wl, m, steps, ms, peak, peak_kind, bool(args.momentum), pipelined=bool(flags))
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         cpu = time_oracle(wl, steps=2, warmup=0, budget_s=20.0, torch_device=dev, all_cores=True)
         cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample", "all_cores") if k in cpu}
 
+    codes = m["codes"]
     line = {"metric": METRIC, "value": units / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "params": wl.num_params, "layers": len(wl.table), "grad_dtype": wl.grad_dtype,
-                       "num_probes": P, "topk_ppm": wl.topk_ppm, "momentum": args.momentum, "weight_decay": args.weight_decay, "parallelism": f"replicas x{world}",
-                       "l2": (f"inputs of one step ({(bytes_in_per_set + state_bytes) / 1e6:.0f} MB) exceed L2 ({l2_bytes / 1e6:.0f} MB)"
-                              if R == 1 else f"{R} rotating buffer sets ({R * (bytes_in_per_set + state_bytes) / 1e6:.0f} MB) exceed L2 ({l2_bytes / 1e6:.0f} MB)"),
+                       "num_probes": P, "topk_ppm": wl.topk_ppm, "t_ctrl": wl.t_ctrl, "momentum": args.momentum,
+                       "weight_decay": args.weight_decay, "flags": flags, "parallelism": f"replicas x{world}", "l2": l2,
                        "codes": {"fp16": codes.count(0), "bf16": codes.count(1), "fp32": codes.count(2)}},
-            "hbm_gbs_algorithmic": step_bytes_min / (ms_step * 1e-3) / 1e9,
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+            "hbm_gbs_algorithmic": roofline["step"]["achieved_gbs"],
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": m["launches"], "clocks": m["clocks"],
+            "configs": configs, "paths": paths}
     print(json.dumps(line))
     D.shutdown()
     return 0
@@ -404,6 +499,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the other configurations and the opt-in paths")
     ap.add_argument("--momentum", type=float, default=0.0)
     ap.add_argument("--weight-decay", type=float, default=0.0)
     ap.add_argument("--t-ctrl", type=int, default=0, help="override the workload's control interval T_ctrl")

@@ -1222,6 +1222,153 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
         if (!A.early_weights || n_slots == 0) start_weight_copies();
         if (bad_seen && lane == 0) atomicMax(A.barrier + 1, A.epoch);
     }
+    // decisions of one layer of this block, from the layer's sums over all blocks (Sec. 3.1 - 3.4).  The new state
+    // replaces the old one in shared memory; the block that holds the layer's first run writes it out once the step
+    // is known to be committed.
+    auto decide = [&](uint32_t q, double pivot, double s1, double s2, uint32_t amax, uint32_t amin) {
+        LayerState st;
+        unsigned long long *words = reinterpret_cast<unsigned long long *>(&st);
+#pragma unroll
+        for (uint32_t i = 0; i < kStateWords; ++i) words[i] = sh_old[q * kStateWords + i];
+        const double n = sh_bl[q].n;
+        const double shift = s1 / n;
+        double var = s2 / n - shift * shift;
+        if (!(var > 0.0)) var = 0.0;
+        LayerScratch sc;
+        sc.mean = pivot + shift; sc.var = var; sc.sum_abs = 0.0; sc.bad = 0ull; sc.amax = amax; sc.amin = amin;
+        uint32_t near;
+        st = decide_layer(A.dp, st, sc, near);
+        sh_eta[q] = st.eta;
+        sh_code[q] = st.code;
+#pragma unroll
+        for (uint32_t i = 0; i < kStateWords; ++i) sh_old[q * kStateWords + i] = words[i];
+    };
+    // a layer's sums over the blocks lo .. hi that share it, in block order, read past L1
+    auto combine_serial = [&](uint32_t q, uint32_t lo, uint32_t hi) {
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+        const double pivot = (double)__ldcg(&A.part[lo].pivot);
+        for (uint32_t i = lo; i < hi; ++i) {
+            const MomentSums m = rebase(__ldcg(&A.part[i].s1), __ldcg(&A.part[i].s2), (double)__ldcg(&A.part[i].n),
+                                        (double)__ldcg(&A.part[i].pivot), pivot);
+            s1 += m.s1;
+            s2 += m.s2;
+            amax = max(amax, __ldcg(&A.part[i].amax));
+            amin = min(amin, __ldcg(&A.part[i].amin));
+        }
+        decide(q, pivot, s1, s2, amax, amin);
+    };
+    auto combine_warp = [&](uint32_t q, uint32_t lo, uint32_t hi) {
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+        const double pivot = (double)__ldcg(&A.part[lo].pivot);
+        for (uint32_t i = lo + lane; i < hi; i += 32) {
+            const MomentSums m = rebase(__ldcg(&A.part[i].s1), __ldcg(&A.part[i].s2), (double)__ldcg(&A.part[i].n),
+                                        (double)__ldcg(&A.part[i].pivot), pivot);
+            s1 += m.s1;
+            s2 += m.s2;
+            amax = max(amax, __ldcg(&A.part[i].amax));
+            amin = min(amin, __ldcg(&A.part[i].amin));
+        }
+        s1 = warp_sum(s1);
+        s2 = warp_sum(s2);
+        amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+        amin = __reduce_min_sync(0xFFFFFFFFu, amin);
+        if (lane == 0) decide(q, pivot, s1, s2, amax, amin);
+    };
+    constexpr uint32_t kThreadCombine = 4;       // layers with at most this many block partials: one thread each
+
+    // update + cast of this warp's slots (Sec. 3.2 step, Sec. 2 master copy and cast)
+    auto walk = [&]() {
+        for (uint32_t s0 = 0; s0 < n_slots; s0 += UA) {
+            float4 wv[UA], gv[UA];
+#pragma unroll
+            for (int u = 0; u < UA; ++u) {
+                const uint32_t s = s0 + u;
+                if (s < n_slots) {
+                    const FusedSlot sl = sh_slot[s];
+                    uint32_t e_lo, e_hi;
+                    lane_range(sl, e_lo, e_hi);
+                    if (e_hi > e_lo) {
+                        const uint64_t i0 = (uint64_t)sl.row * 128ull + lane * 4u;
+                        wv[u] = s < A.cap_w ? sh_w[s * 32u + lane] : ld_stream(A.w + i0);
+                        gv[u] = s < A.cap_g ? sh_g[s * 32u + lane] : GradVec<BF16>::load4(A.g, i0, true);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UA; ++u) {
+                const uint32_t s = s0 + u;
+                if (s < n_slots) {
+                    const FusedSlot sl = sh_slot[s];
+                    uint32_t e_lo, e_hi;
+                    lane_range(sl, e_lo, e_hi);
+                    if (e_hi > e_lo) {
+                        const uint64_t i0 = (uint64_t)sl.row * 128ull + lane * 4u;
+                        const uint32_t code = sh_code[sl.seg - lf];
+                        float4 x = wv[u];
+                        const float neg_eta = -sh_eta[sl.seg - lf];
+                        x.x = fmaf(neg_eta, gv[u].x, x.x);
+                        x.y = fmaf(neg_eta, gv[u].y, x.y);
+                        x.z = fmaf(neg_eta, gv[u].z, x.z);
+                        x.w = fmaf(neg_eta, gv[u].w, x.w);
+                        if (e_lo == 0u && e_hi == 4u) {
+                            __stcs(reinterpret_cast<float4 *>(A.w + i0), x);
+                            {
+                                if (code == 0u) {
+                                    const __half2 a = __floats2half2_rn(x.x, x.y), b = __floats2half2_rn(x.z, x.w);
+                                    uint2 o;
+                                    o.x = *reinterpret_cast<const uint32_t *>(&a);
+                                    o.y = *reinterpret_cast<const uint32_t *>(&b);
+                                    __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
+                                } else if (code == 1u) {
+                                    const __nv_bfloat162 a = __floats2bfloat162_rn(x.x, x.y), b = __floats2bfloat162_rn(x.z, x.w);
+                                    uint2 o;
+                                    o.x = *reinterpret_cast<const uint32_t *>(&a);
+                                    o.y = *reinterpret_cast<const uint32_t *>(&b);
+                                    __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
+                                }
+                            }
+                        } else {
+                            // a vector on the edge of the layer: only the elements of this run are written
+                            const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                            for (uint32_t e = 0; e < 4; ++e) {
+                                if (e >= e_lo && e < e_hi) {
+                                    A.w[i0 + e] = xs[e];
+                                    if (code < 2u) A.c[i0 + e] = cast16(xs[e], code);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    };
+    // the step's status; a skipped step changes nothing and block 0 sums the exact count of non-finite values
+    auto write_status = [&](bool skip) {
+        if (blockIdx.x == 0 && tid == 0) {
+            A.status->step = A.step;
+            A.status->skipped = skip ? 1u : 0u;
+            if (!skip) A.status->nonfinite = 0ull;
+        }
+        if (skip && blockIdx.x == 0) {
+            __shared__ double red[kWarps];
+            double total = 0.0;
+            for (uint32_t i = tid; i < A.n_part; i += kThreads) total += (double)__ldcg(&A.part[i].bad);
+            total = block_sum(total, red);
+            if (tid == 0) A.status->nonfinite = (unsigned long long)total;
+        }
+    };
+    auto commit_states = [&]() {
+        for (uint32_t q = tid; q < nl; q += kThreads) {
+            if (!sh_bl[q].own) continue;
+            unsigned long long *dst = reinterpret_cast<unsigned long long *>(A.state + lf + q);
+#pragma unroll
+            for (uint32_t i = 0; i < kStateWords; ++i) dst[i] = sh_old[q * kStateWords + i];
+        }
+    };
+
     // the block's runs folded into one partial per layer it touches, in run order
     cp_async_wait_but_one();        // the block's tables have arrived (the weight copies may still be under way)
     __syncthreads();
@@ -1246,145 +1393,21 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
 
     // did any warp of the grid see a non-finite input?  The answer is needed only when results are committed, so
     // the decisions below are taken while it is on its way; those of a skipped step are thrown away
-    const bool skip = __ldcg(A.barrier + 1) == A.epoch;
-
-    // decisions of the layers this block touches, from the block partials of each (Sec. 3.1 - 3.4)
-    auto decide = [&](uint32_t q, double pivot, double s1, double s2, uint32_t amax, uint32_t amin) {
-        LayerState old;
-        unsigned long long *dst = reinterpret_cast<unsigned long long *>(&old);
-#pragma unroll
-        for (uint32_t i = 0; i < kStateWords; ++i) dst[i] = sh_old[q * kStateWords + i];
-        const double n = sh_bl[q].n;
-        const double shift = s1 / n;
-        double var = s2 / n - shift * shift;
-        if (!(var > 0.0)) var = 0.0;
-        LayerScratch sc;
-        sc.mean = pivot + shift; sc.var = var; sc.sum_abs = 0.0; sc.bad = 0ull; sc.amax = amax; sc.amin = amin;
-        uint32_t near;
-        const LayerState st = decide_layer(A.dp, old, sc, near);
-        sh_eta[q] = st.eta;
-        sh_code[q] = st.code;
-        if (sh_bl[q].own && !skip) A.state[lf + q] = st;
-    };
-    constexpr uint32_t kThreadCombine = 4;       // layers with at most this many block partials: one thread each
+    const bool skip = __ldcg(A.barrier + 1) == A.epoch || __ldcg(&A.status->device_error) != 0u;
     for (uint32_t q = tid; q < nl; q += kThreads) {
         const uint32_t lo = sh_bl[q].part_lo, hi = sh_bl[q].part_hi;
-        if (hi - lo > kThreadCombine) continue;
-        double s1 = 0.0, s2 = 0.0;
-        uint32_t amax = 0u, amin = 0xFFFFFFFFu;
-        const double pivot = (double)__ldcg(&A.part[lo].pivot);
-        for (uint32_t i = lo; i < hi; ++i) {
-            const MomentSums m = rebase(__ldcg(&A.part[i].s1), __ldcg(&A.part[i].s2), (double)__ldcg(&A.part[i].n),
-                                        (double)__ldcg(&A.part[i].pivot), pivot);
-            s1 += m.s1;
-            s2 += m.s2;
-            amax = max(amax, __ldcg(&A.part[i].amax));
-            amin = min(amin, __ldcg(&A.part[i].amin));
-        }
-        decide(q, pivot, s1, s2, amax, amin);
+        if (hi - lo <= kThreadCombine) combine_serial(q, lo, hi);
     }
     for (uint32_t q = warp; q < nl; q += kWarps) {      // layers spread over many blocks: one warp each
         const uint32_t lo = sh_bl[q].part_lo, hi = sh_bl[q].part_hi;
-        if (hi - lo <= kThreadCombine) continue;
-        double s1 = 0.0, s2 = 0.0;
-        uint32_t amax = 0u, amin = 0xFFFFFFFFu;
-        const double pivot = (double)__ldcg(&A.part[lo].pivot);
-        for (uint32_t i = lo + lane; i < hi; i += 32) {
-            const MomentSums m = rebase(__ldcg(&A.part[i].s1), __ldcg(&A.part[i].s2), (double)__ldcg(&A.part[i].n),
-                                        (double)__ldcg(&A.part[i].pivot), pivot);
-            s1 += m.s1;
-            s2 += m.s2;
-            amax = max(amax, __ldcg(&A.part[i].amax));
-            amin = min(amin, __ldcg(&A.part[i].amin));
-        }
-        s1 = warp_sum(s1);
-        s2 = warp_sum(s2);
-        amax = __reduce_max_sync(0xFFFFFFFFu, amax);
-        amin = __reduce_min_sync(0xFFFFFFFFu, amin);
-        if (lane == 0) decide(q, pivot, s1, s2, amax, amin);
+        if (hi - lo > kThreadCombine) combine_warp(q, lo, hi);
     }
     cp_async_wait_all();
-    if (blockIdx.x == 0 && tid == 0) {
-        A.status->step = A.step;
-        A.status->skipped = skip ? 1u : 0u;
-        if (!skip) A.status->nonfinite = 0ull;
-    }
-    if (skip) {
-        // skipped step: nothing changes.  The exact count of non-finite values is summed by block 0.
-        if (blockIdx.x == 0) {
-            __shared__ double red[kWarps];
-            double total = 0.0;
-            for (uint32_t i = tid; i < A.n_part; i += kThreads) total += (double)__ldcg(&A.part[i].bad);
-            total = block_sum(total, red);
-            if (tid == 0) A.status->nonfinite = (unsigned long long)total;
-        }
-        return;
-    }
+    write_status(skip);
+    if (skip) return;
     __syncthreads();
-
-    // phase 2: update + cast of this warp's slots (Sec. 3.2 step, Sec. 2 master copy and cast)
-    for (uint32_t s0 = 0; s0 < n_slots; s0 += UA) {
-        float4 wv[UA], gv[UA];
-#pragma unroll
-        for (int u = 0; u < UA; ++u) {
-            const uint32_t s = s0 + u;
-            if (s < n_slots) {
-                const FusedSlot sl = sh_slot[s];
-                uint32_t e_lo, e_hi;
-                lane_range(sl, e_lo, e_hi);
-                if (e_hi > e_lo) {
-                    const uint64_t i0 = (uint64_t)sl.row * 128ull + lane * 4u;
-                    wv[u] = s < A.cap_w ? sh_w[s * 32u + lane] : ld_stream(A.w + i0);
-                    gv[u] = s < A.cap_g ? sh_g[s * 32u + lane] : GradVec<BF16>::load4(A.g, i0, true);
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < UA; ++u) {
-            const uint32_t s = s0 + u;
-            if (s < n_slots) {
-                const FusedSlot sl = sh_slot[s];
-                uint32_t e_lo, e_hi;
-                lane_range(sl, e_lo, e_hi);
-                if (e_hi > e_lo) {
-                    const uint64_t i0 = (uint64_t)sl.row * 128ull + lane * 4u;
-                    const float neg_eta = -sh_eta[sl.seg - lf];
-                    const uint32_t code = sh_code[sl.seg - lf];
-                    float4 x = wv[u];
-                    x.x = fmaf(neg_eta, gv[u].x, x.x);
-                    x.y = fmaf(neg_eta, gv[u].y, x.y);
-                    x.z = fmaf(neg_eta, gv[u].z, x.z);
-                    x.w = fmaf(neg_eta, gv[u].w, x.w);
-                    if (e_lo == 0u && e_hi == 4u) {
-                        __stcs(reinterpret_cast<float4 *>(A.w + i0), x);
-                        if (code == 0u) {
-                            const __half2 a = __floats2half2_rn(x.x, x.y), b = __floats2half2_rn(x.z, x.w);
-                            uint2 o;
-                            o.x = *reinterpret_cast<const uint32_t *>(&a);
-                            o.y = *reinterpret_cast<const uint32_t *>(&b);
-                            __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
-                        } else if (code == 1u) {
-                            const __nv_bfloat162 a = __floats2bfloat162_rn(x.x, x.y), b = __floats2bfloat162_rn(x.z, x.w);
-                            uint2 o;
-                            o.x = *reinterpret_cast<const uint32_t *>(&a);
-                            o.y = *reinterpret_cast<const uint32_t *>(&b);
-                            __stcs(reinterpret_cast<uint2 *>(A.c + i0), o);
-                        }
-                    } else {
-                        // a vector on the edge of the layer: only the elements of this run are written
-                        const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                        for (uint32_t e = 0; e < 4; ++e) {
-                            if (e >= e_lo && e < e_hi) {
-                                A.w[i0 + e] = xs[e];
-                                if (code < 2u) A.c[i0 + e] = cast16(xs[e], code);
-                            }
-                        }
-                    }
-                }
-            }
-        }
-    }
+    commit_states();
+    walk();
 }
 
 // ------------------------------------------------------------------ power iteration support (Sec. 3.2)

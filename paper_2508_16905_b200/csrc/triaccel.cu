@@ -388,6 +388,7 @@ int check_device_error(ta_handle *h)
     s.device_error = 0u;
     TA_CUDA(h, cudaMemcpy(h->d.status, &s, sizeof(s), cudaMemcpyHostToDevice));
     if (h->d.barrier) TA_CUDA(h, cudaMemset(h->d.barrier, 0, 2 * sizeof(unsigned long long)));
+
     h->barrier_base = 0;
     h->fused_launches = 0;
     if (h->pipe_ok) {
@@ -631,6 +632,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     if (h->fused_ok) {
         TA_TRY(dev_alloc(&d.barrier, 2));
         TA_TRY(cudaMemset(d.barrier, 0, 2 * sizeof(unsigned long long)));
+
         TA_TRY(dev_alloc(&d.warp_head, run_plan.warp_head.size()));
         TA_TRY(cudaMemcpy(d.warp_head, run_plan.warp_head.data(), run_plan.warp_head.size() * sizeof(ta::FusedWarpHead), cudaMemcpyHostToDevice));
         TA_TRY(dev_alloc(&d.block_head, run_plan.block_head.size()));
@@ -873,7 +875,8 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
         fa.max_slots = h->fused_slots; fa.max_block_runs = h->fused_block_runs; fa.max_block_layers = h->fused_block_layers;
         fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base;
         fa.epoch = h->fused_launches + 1;
-        fa.early_weights = 0u;      // the weight copies start after the sweep (measured faster than starting them with its first loads)
+        fa.early_weights = 0u;
+      // the weight copies start after the sweep (measured faster than starting them with its first loads)
         if (h->expire_next_wait) { fa.barrier_base += 1ull << 40; h->expire_next_wait = false; }
         const int grid = h->fused_grid;
         void *args[] = {&fa};
