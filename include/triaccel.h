@@ -209,8 +209,10 @@ int ta_precision_codes(ta_handle *h, uint8_t *out_host);
  * ta_masks -- the top-k mask of the last step with Hz: bit (i & 31) of word i >> 5 is set when
  * flat element i is among the k_l largest |S| of its layer (ties: lower index first); bits of
  * gaps are 0.  *dev_bits is library-owned device memory, valid until the next ta_step with Hz or
- * ta_destroy; read it on the stream used for ta_step.  With topk_ppm == 1000000 every element is
- * in the mask, nothing is stored, and *dev_bits = NULL, *num_words = 0.
+ * ta_destroy; read it on the stream used for ta_step.  The library keeps two mask buffers that swap roles
+ * whenever a step with Hz commits, so call ta_masks again after such a step; the call waits for the stream of
+ * the last ta_step.  With topk_ppm == 1000000 every element is in the mask, nothing is stored, and
+ * *dev_bits = NULL, *num_words = 0.
  */
 int ta_masks(ta_handle *h, const uint32_t **dev_bits, uint64_t *num_words);
 
@@ -241,6 +243,40 @@ int ta_power_iterate(ta_handle *h, const float *u, const float *Hu, const float 
  * Errors: TA_ERR_ARG (NULL, negative or non-finite value), TA_ERR_CUDA.
  */
 int ta_set_curvature(ta_handle *h, const float *lambda_max_host);
+
+/*
+ * A model spread over several GPUs by flat ranges (the paper leaves multi-GPU training as future work, Sec. 4.5; this
+ * is the optimizer pass's side of it).  Rank r holds the elements [range_lo, range_hi) of every flat buffer, which may
+ * cut layers anywhere on a multiple of 128 elements.  All decisions of the pass are per layer and need only the
+ * layer's sums (Sec. 3.1: mean and variance; Sec. 3.2: the largest |S|), so one small exchange per step is enough:
+ *
+ *   ta_shard_sweep   statistics of the local part of every layer, one ta_layer_record per layer (device memory)
+ *   (the caller gathers the records of all ranks, in rank order: world * L records; e.g. an NCCL all-gather)
+ *   ta_shard_apply   combines the records in rank order (every rank arrives at identical numbers), takes the
+ *                    decisions, screens the step (a non-finite value on any rank skips the step on every rank) and
+ *                    updates the local weights and copies
+ *
+ * ta_create_shard takes the table and n_total of the WHOLE model plus this rank's range; the buffers passed to the two
+ * calls hold only the range (element i of the model at index i - range_lo; Hz_local is [P][range_hi - range_lo]).
+ * The probes are those of the whole model (they depend on the flat index, not on the cut).  Results equal those of
+ * one handle over the whole model: codes, step sizes, weights and copies bit for bit, the double-precision moments up
+ * to the order of summation.  Dense curvature only (topk_ppm == 1000000), no momentum buffer; ta_stats, ta_set_lr,
+ * ta_precision_codes and the state calls work as usual (every rank holds the state of all layers); ta_step returns
+ * TA_ERR_STATE on such a handle.
+ */
+typedef struct ta_layer_record {
+    double s1, s2;        /* sums of (g - pivot) and (g - pivot)^2 over the local elements of the layer */
+    double n;             /* their number (0: the layer has no element on this rank)                     */
+    float pivot;          /* the first local gradient value of the layer                                 */
+    uint32_t amax, amin;  /* largest / smallest |S| (bit patterns)                                       */
+    uint32_t bad;         /* non-finite inputs                                                           */
+} ta_layer_record;
+int ta_create_shard(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hparams *hp, uint64_t range_lo,
+                    uint64_t range_hi, ta_handle **out);
+int ta_shard_sweep(ta_handle *h, const void *g_local, const float *Hz_local, uint64_t probe_seed, uint64_t step,
+                   ta_layer_record *records_out /* device, L records */, void *stream);
+int ta_shard_apply(ta_handle *h, float *w_local, const void *g_local, uint16_t *c_local,
+                   const ta_layer_record *records_all /* device, world * L records, rank-major */, uint32_t world, void *stream);
 
 /* Number of kernels the library launched on behalf of this handle so far (for benchmarks). */
 int ta_launch_count(ta_handle *h, uint64_t *count);

@@ -22,7 +22,8 @@ EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "t
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
            "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
            "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait",
-           "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch", "ta_plan_pipeline"]
+           "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch", "ta_plan_pipeline",
+           "ta_create_shard", "ta_shard_sweep", "ta_shard_apply"]
 
 
 class ta_segment(C.Structure):
@@ -110,6 +111,9 @@ def lib():
     L.ta_plan_one_launch.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_run), u32, C.POINTER(u32), C.POINTER(u32),
                                      C.POINTER(u32)]
     L.ta_plan_pipeline.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_task), u64, C.POINTER(u64)]
+    L.ta_create_shard.argtypes = [C.POINTER(ta_segment), u32, u64, C.POINTER(ta_hparams), u64, u64, C.POINTER(vp)]
+    L.ta_shard_sweep.argtypes = [vp, vp, vp, u64, u64, vp, vp]
+    L.ta_shard_apply.argtypes = [vp, vp, vp, vp, vp, u32, vp]
     L.ta_static_last_error.argtypes = []
     L.ta_static_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -181,6 +185,33 @@ def ta_create(table, n_total, hp=None, **hp_kwargs):
     if rc != TA_OK:
         raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
     return Handle(out, L, int(n_total), hp)
+
+
+RECORD_BYTES = 40          # sizeof(ta_layer_record)
+
+
+def ta_create_shard(table, n_total, range_lo, range_hi, hp=None, **hp_kwargs):
+    """A handle for the flat range [range_lo, range_hi) of a model spread over ranks; table and n_total are the whole model's."""
+    hp = hp if hp is not None else make_hparams(**hp_kwargs)
+    L = len(table)
+    segs = (ta_segment * max(L, 1))(*[ta_segment(int(o), int(n)) for o, n in table])
+    out = C.c_void_p()
+    rc = lib().ta_create_shard(segs, L, int(n_total), C.byref(hp), int(range_lo), int(range_hi), C.byref(out))
+    if rc != TA_OK:
+        raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
+    return Handle(out, L, int(n_total), hp)
+
+
+def ta_shard_sweep(h, g_local, Hz_local, probe_seed, step, records_out, stream=None):
+    """records_out: CUDA uint8 tensor of L * RECORD_BYTES bytes (8-byte aligned)."""
+    _check(lib().ta_shard_sweep(h.ptr, _dev_ptr(g_local), _dev_ptr(Hz_local), int(probe_seed), int(step),
+                                _dev_ptr(records_out), _stream(stream)), h.ptr)
+
+
+def ta_shard_apply(h, w_local, g_local, c_local, records_all, world, stream=None):
+    """records_all: CUDA uint8 tensor of world * L * RECORD_BYTES bytes, the ranks' records in rank order."""
+    _check(lib().ta_shard_apply(h.ptr, _dev_ptr(w_local), _dev_ptr(g_local), _dev_ptr(c_local), _dev_ptr(records_all),
+                                int(world), _stream(stream)), h.ptr)
 
 
 def ta_destroy(h):

@@ -85,18 +85,32 @@ struct Status {
     unsigned long long step, nonfinite;
     uint32_t skipped, near_count;
     uint32_t done_counter, device_error;   // device_error: a bounded wait inside a kernel ran out
-    uint32_t near_stage, pad;              // near-threshold layers of a step that may still be skipped
+    uint32_t mask_cur;                     // top-k: which of the two mask buffers holds the current mask
+    uint32_t redo_layers;                  // top-k: layers of this step whose guessed selection window missed
 };
 
 // Per-layer bookkeeping of the radix select.
 struct SelectState {
-    uint32_t prefix;      // bits of the threshold fixed so far
-    uint32_t remaining;   // how many elements are still to be taken inside the prefix
+    uint32_t prefix;      // level-1 bin (bits 30..20 of |S|) of the layer's k-th largest |S|
+    uint32_t remaining;   // how many elements are still to be taken inside that bin
     uint32_t thr_bits;    // final threshold bit pattern
     uint32_t take_equal;  // how many elements equal to the threshold belong to the mask
     uint32_t surplus;     // 1: more elements equal the threshold than are taken (index tie-break needed)
+    uint32_t valid;       // 1: the window the sweep collected candidates in contains the bin
+    uint32_t lo_bin;      // lowest bin the layer's candidate list holds
     uint32_t pad;
 };
+
+// What one rank of a sharded pass knows about a layer after its sweep: the sums over the elements it holds, taken
+// around its first gradient value of the layer.  Ranks exchange these records and every rank combines them in rank order.
+struct LayerRecord {
+    double s1, s2;        // sums of (g - pivot) and (g - pivot)^2
+    double n;             // elements of the layer on this rank (0: none, the other fields are then ignored)
+    float pivot;
+    uint32_t amax, amin;  // largest / smallest |S| as bit patterns
+    uint32_t bad;         // non-finite inputs
+};
+static_assert(sizeof(LayerRecord) == 40, "the record is part of the C ABI (ta_layer_record)");
 
 struct Hyper {
     float beta, tau_low, tau_high, tau_curv, alpha;
@@ -244,13 +258,59 @@ struct SweepArgs {
     double *p_s1, *p_s2, *p_sa;
     float *p_piv;
     uint32_t *p_amax, *p_amin, *p_bad;
-    // top-k only
-    float *abs_s;             // [n_total] |S|
+    // top-k only.  The sweep selects as it goes: from the last step with curvature it knows, per layer, a window of
+    // level-1 bins (bits 30..20 of |S|) in which the k-th largest |S| should fall again.  Elements above the window get
+    // their mask bit at once, elements inside it are listed as candidates, and the level-1 histogram tells afterwards
+    // whether the window held.  Where it did not (or there was none: the first step), a second launch with redo = 1
+    // repeats the layer with the exact bin.  All of it goes to the mask buffer that is not current; the buffers swap
+    // roles when the step commits.
     uint32_t *hist;           // [L][kHistBins], level-1 histogram of |S| bit patterns
     const uint32_t *batch_seg; // [n_batches] layer of a batch whose items all lie in one layer, else kMixedBatch
+    uint32_t *mask2;          // two buffers of mask_words words
+    uint64_t mask_words;
+    const uint2 *window;      // [L] lowest and highest bin of the window (lowest > highest: no guess)
+    const SelectState *sel;   // [L] redo: the exact bin and whether the layer needs the second pass
+    uint32_t *cand_count;     // [L]
+    uint32_t *cand_val;       // [n_total], candidates of layer l at seg_off[l] ...
+    uint32_t *cand_idx;       // [n_total]
+    const uint64_t *seg_off;  // [L]
+    double *p_mass;           // per item: sum of |S| above the window
+    const Status *status;
+    uint32_t redo;
 };
 
 constexpr uint32_t kMixedBatch = 0xFFFFFFFFu;
+
+constexpr uint32_t kStageCap = 384;      // candidates a warp collects in shared memory before it reserves list slots
+
+// Stages this lane's candidates (bit e of `cand` = element e of its vector) in the warp's shared-memory
+// buffer, behind the `running` ones already there.  Whole warp; `running` stays warp-uniform.
+__device__ __forceinline__ void stage_candidates(uint32_t cand, const uint32_t (&ab)[4], uint32_t local0, uint32_t lane,
+                                                 uint32_t &running, uint32_t *sval, uint32_t *sidx)
+{
+    if (!__any_sync(0xFFFFFFFFu, cand != 0u)) return;
+    const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+    for (uint32_t e = 0; e < 4; ++e) {
+        const uint32_t who = __ballot_sync(0xFFFFFFFFu, (cand >> e) & 1u);
+        if ((cand >> e) & 1u) {
+            const uint32_t pos = running + (uint32_t)__popc(who & below);
+            sval[pos] = ab[e];
+            sidx[pos] = local0 + e;
+        }
+        running += (uint32_t)__popc(who);
+    }
+}
+
+// 8 lanes make one 32-bit mask word out of their 4-bit pieces.
+__device__ __forceinline__ uint32_t gather_word(uint32_t nib, uint32_t lane)
+{
+    uint32_t word = nib << ((lane & 7u) * 4u);
+    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+    return word;
+}
 
 template <int P> struct RowData {
     float4 g;
@@ -364,7 +424,8 @@ struct ItemSums {
 // of the rows it sweeps (with the step size and code the layers had before this step) and writes their 16-bit copies.
 template <int P, bool BF16, bool TOPK, bool APPLY, int ROWS = 0, typename Store>
 __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, uint32_t *sh_hist, const Store &store,
-                                            const SinglePass &sp = SinglePass{nullptr, nullptr, nullptr, 0.f})
+                                            const SinglePass &sp = SinglePass{nullptr, nullptr, nullptr, 0.f},
+                                            uint32_t *sh_stage = nullptr /* TOPK: [kWarps][2][kStageCap] */)
 {
     static_assert(!(APPLY && TOPK), "the single-pass variant is for dense curvature");
     constexpr int PP = P > 0 ? P : 1;
@@ -383,9 +444,24 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                 for (uint32_t b = threadIdx.x; b < (uint32_t)kHistBins; b += kThreads) sh_hist[b] = 0u;
             __syncthreads();
         }
-        const Item item = it < A.n_items ? A.items[it] : Item{0, 0, 0};
-        if (it < A.n_items && item.len == 0u && lane == 0)     // padding item: neutral partials
+        Item item = it < A.n_items ? A.items[it] : Item{0, 0, 0};
+        if (it < A.n_items && item.len == 0u && lane == 0) {   // padding item: neutral partials
             store(it, ItemSums{0.0, 0.0, 0.0, 0.f, 0u, 0u, 0xFFFFFFFFu, 0u});
+            if (TOPK) A.p_mass[it] = 0.0;
+        }
+        // top-k: the window of level-1 bins this pass works with, and whether it touches the mask at all
+        uint32_t win_lo = 1u, win_hi = 0u;
+        if (TOPK && item.len != 0u) {
+            if (A.redo) {
+                const SelectState ss = A.sel[item.seg];
+                if (ss.valid) item.len = 0u;                   // the first pass got this layer right
+                win_lo = win_hi = ss.prefix;
+            } else {
+                const uint2 win = A.window[item.seg];
+                win_lo = win.x; win_hi = win.y;
+            }
+        }
+        const bool masking = TOPK && win_lo <= win_hi;
         if (item.len != 0u) {
         const uint64_t begin = item.begin, end = begin + item.len;
         const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
@@ -399,8 +475,60 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             code = sp.state[item.seg].code;
         }
         auto hist_add = [&](uint32_t ab) {
+            if (A.redo) return;
             if (uniform) atomicAdd(&sh_hist[ab >> 20], 1u);
             else atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
+        };
+        // top-k: mask bits above the window, candidates inside it
+        const uint64_t seg_b = TOPK ? A.seg_off[item.seg] : 0ull;
+        uint32_t *mask = TOPK ? A.mask2 + (size_t)(A.redo ? A.status->mask_cur : 1u - A.status->mask_cur) * A.mask_words : nullptr;
+        uint32_t *sval = TOPK ? sh_stage + (size_t)warp * 2u * kStageCap : nullptr, *sidx = TOPK ? sval + kStageCap : nullptr;
+        uint32_t staged = 0u;
+        double mass = 0.0;
+        // moves the staged candidates to the layer's list: one slot reservation for all of them
+        auto flush = [&]() {
+            if (staged == 0u) return;
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(A.cand_count + item.seg, staged);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            __syncwarp();
+            for (uint32_t j = lane; j < staged; j += 32) {
+                A.cand_val[seg_b + base + j] = sval[j];
+                A.cand_idx[seg_b + base + j] = sidx[j];
+            }
+            __syncwarp();
+            staged = 0u;
+        };
+        // one row: ab = |S| patterns of this lane's four elements, inside = which of them belong to the item
+        auto mask_row = [&](uint64_t row, const uint32_t (&ab)[4], uint32_t inside, bool whole) {
+            uint32_t nib = 0u, cand = 0u;
+            float above = 0.f;
+#pragma unroll
+            for (uint32_t e = 0; e < 4; ++e) {
+                const uint32_t bin = ab[e] >> 20;
+                if ((inside >> e) & 1u) {
+                    if (bin > win_hi) { nib |= 1u << e; above += __uint_as_float(ab[e]); }
+                    else if (bin >= win_lo) cand |= 1u << e;
+                }
+            }
+            mass += (double)above;
+            if (staged + 128u > kStageCap) flush();
+            stage_candidates(cand, ab, (uint32_t)(row * 128ull - seg_b) + lane * 4u, lane, staged, sval, sidx);
+            const uint32_t word = gather_word(nib, lane);
+            if ((lane & 7u) == 0u) {
+                const uint64_t w0 = row * 128ull + (lane >> 3) * 32ull;     // first element of this word
+                uint32_t *dst = mask + (w0 >> 5);
+                if (whole || (w0 >= begin && w0 + 32u <= end)) {
+                    *dst = word;
+                } else if (w0 + 32u > begin && w0 < end) {
+                    // the other bits of this word belong to a neighbouring layer or a gap: replace only ours
+                    const uint32_t lo_bit = begin > w0 ? (uint32_t)(begin - w0) : 0u;
+                    const uint32_t hi_bit = end < w0 + 32u ? (uint32_t)(end - w0) : 32u;     // exclusive
+                    const uint32_t ours = (hi_bit == 32u ? 0xFFFFFFFFu : ((1u << hi_bit) - 1u)) & ~((1u << lo_bit) - 1u);
+                    atomicAnd(dst, ~ours);
+                    if (word) atomicOr(dst, word);
+                }
+            }
         };
         uint32_t X[PP][4];
         uint64_t have_block = ~0ull;
@@ -424,6 +552,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
 #pragma unroll
             for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
             const uint64_t i0 = row * 128ull + lane * 4u;
+            uint32_t abs4[4] = {0u, 0u, 0u, 0u}, inside = 0u;
 #pragma unroll
             for (uint32_t e = 0; e < 4; ++e) {
                 const uint64_t i = i0 + e;
@@ -433,18 +562,20 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                     for (int p = 0; p < PP; ++p) hv[p] = (P > 0) ? __ldcs(A.hz + (uint64_t)p * A.n_total + i) : 0.f;
                     const float gv = GradVec<BF16>::load1(A.g, i);
                     const uint32_t ab = acc.element(gv, hv, sel, (k & 7u) * 4u + e);
+                    abs4[e] = ab;
+                    inside |= 1u << e;
                     if (APPLY) {
                         const float wn = fmaf(neg_eta, gv, sp.w[i]);
                         sp.w[i] = wn;
                         if (code < 2u) sp.c[i] = cast16(wn, code);
                     }
-                    if (TOPK) {
-                        A.abs_s[i] = __uint_as_float(ab);
-                        hist_add(ab);
-                    }
+                    if (TOPK) hist_add(ab);
                 }
             }
-            if (TOPK) acc.end_row();
+            if (TOPK) {
+                acc.end_row();
+                if (masking) mask_row(row, abs4, inside, false);
+            }
         };
 
         auto full_rows = [&](uint64_t row, RowData<P> (&rd)[U], int count) {
@@ -456,7 +587,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
 #pragma unroll
                     for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
                     const float gv[4] = {rd[u].g.x, rd[u].g.y, rd[u].g.z, rd[u].g.w};
-                    float av[4];
+                    uint32_t abs4[4];
 #pragma unroll
                     for (uint32_t e = 0; e < 4; ++e) {
                         float hv[PP];
@@ -466,13 +597,22 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                             hv[p] = e == 0 ? h.x : (e == 1 ? h.y : (e == 2 ? h.z : h.w));
                         }
                         const uint32_t ab = acc.element(gv[e], hv, sel, (k & 7u) * 4u + e);
-                        av[e] = __uint_as_float(ab);
-                        if (TOPK) hist_add(ab);
+                        abs4[e] = ab;
                     }
                     if (TOPK) {
+                        // exact zeros (pruned or untouched weights) would all hit one counter: the warp counts them together
+                        uint32_t zeros = 0u;
+#pragma unroll
+                        for (uint32_t e = 0; e < 4; ++e) {
+                            zeros += (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, abs4[e] == 0u));
+                            if (abs4[e] != 0u) hist_add(abs4[e]);
+                        }
+                        if (lane == 0 && zeros != 0u && !A.redo) {
+                            if (uniform) atomicAdd(&sh_hist[0], zeros);
+                            else atomicAdd(A.hist + (uint64_t)item.seg * kHistBins, zeros);
+                        }
                         acc.end_row();
-                        const uint64_t i0 = (row + u) * 128ull + lane * 4u;
-                        *reinterpret_cast<float4 *>(A.abs_s + i0) = make_float4(av[0], av[1], av[2], av[3]);
+                        if (masking) mask_row(row + u, abs4, 0xFu, true);
                     }
                     if (APPLY) update_store4<true>(sp.w, sp.c, (row + u) * 128ull + lane * 4u, rd[u].w, rd[u].g, neg_eta, code);
                 }
@@ -543,6 +683,11 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             bad = __reduce_add_sync(0xFFFFFFFFu, bad);
         }
         if (lane == 0) store(it, ItemSums{s1, s2, sa, piv, item.len, amax, amin, bad});
+        if (masking) {
+            flush();
+            mass = warp_sum(mass);
+            if (lane == 0) A.p_mass[it] = mass;
+        }
         }   // item.len != 0
         if (TOPK) {
             __syncthreads();
@@ -560,6 +705,8 @@ template <int P, bool BF16, bool TOPK>
 __global__ void __launch_bounds__(kThreads, (P == 4 ? TA_SWEEP_MIN_BLOCKS_P4 : 1)) k_sweep(const SweepArgs A)
 {
     __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
+    __shared__ uint32_t sh_stage[TOPK ? kWarps * 2 * kStageCap : 1];
+    if (TOPK && A.redo && (A.status->skipped || A.status->redo_layers == 0u)) return;      // nothing to repeat
     auto store = [&A](uint32_t it, const ItemSums &r) {
         A.p_s1[it] = r.s1;
         A.p_s2[it] = r.s2;
@@ -568,7 +715,7 @@ __global__ void __launch_bounds__(kThreads, (P == 4 ? TA_SWEEP_MIN_BLOCKS_P4 : 1
         if (P > 0) { A.p_amax[it] = r.amax; A.p_amin[it] = r.amin; }
         if (TOPK) A.p_sa[it] = r.sa;
     };
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK, false>(A, batch, sh_hist, store);
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK, false>(A, batch, sh_hist, store, SinglePass{nullptr, nullptr, nullptr, 0.f}, sh_stage);
 }
 
 // ------------------------------------------------------------------ decisions
@@ -637,6 +784,8 @@ struct DecideArgs {
     SelectState *sel;
     uint32_t *cand_count;
     const uint64_t *seg_k;
+    uint2 *window;                  // [L] the bins the sweep collected candidates in; rewritten for the next step
+    LayerRecord *record_out;        // sharded pass: [L] this rank's sums per layer are written here and nothing is decided
 };
 
 // Reads another block's results past the L1 cache (they were published with a fence).
@@ -696,6 +845,31 @@ __device__ __forceinline__ uint32_t commit_layer(const DecideArgs &A, uint32_t l
     return near;
 }
 
+// Whole block: screens the step for non-finite input over all layers and, if it is clean, commits every layer
+// (EMAs, codes, step sizes); writes the step's status.
+__device__ __forceinline__ void commit_step(const DecideArgs &A, double *red)
+{
+    const uint32_t tid = threadIdx.x;
+    double total_bad = 0.0;
+    for (uint32_t j = tid; j < A.L; j += kThreads)
+        total_bad += (double)__ldcg(&A.scratch[j].bad);
+    total_bad = block_sum(total_bad, red);
+    double near = 0.0;
+    if (total_bad == 0.0)
+        for (uint32_t j = tid; j < A.L; j += kThreads) near += (double)commit_layer(A, j);
+    near = block_sum(near, red);
+    if (A.topk && total_bad != 0.0)          // a skipped step: what the sweep listed is of no use
+        for (uint32_t j = tid; j < A.L; j += kThreads) A.cand_count[j] = 0u;
+    if (tid == 0) {
+        A.status->step = A.step;
+        A.status->nonfinite = (unsigned long long)total_bad;
+        A.status->skipped = total_bad != 0.0 ? 1u : 0u;
+        if (A.control && total_bad == 0.0) A.status->near_count = (uint32_t)near;
+        if (A.topk && total_bad == 0.0) A.status->mask_cur ^= 1u;       // the buffer the sweep wrote becomes the mask
+        A.status->done_counter = 0u;
+    }
+}
+
 // One block per layer combines the layer's item partials in a fixed order; the block that
 // finishes last screens the whole step for non-finite input and commits every layer.
 __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
@@ -721,23 +895,40 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
         const uint32_t k = (uint32_t)A.seg_k[l];
         block_find_bin<true>(h, kHistBins, k, scan, found);
         if (tid == 0) {
+            // did the window the sweep worked with contain the bin?  If not, its candidates are dropped and the layer
+            // is repeated with the exact bin.  Either way the next step starts from a window around this bin.
+            const uint2 win = A.window[l];
             SelectState s;
             s.prefix = found[0];
             s.remaining = k - found[1];
             s.thr_bits = 0u; s.take_equal = 0u; s.surplus = 0u; s.pad = 0u;
+            s.valid = (win.x <= win.y && win.x <= found[0] && found[0] <= win.y) ? 1u : 0u;
+            s.lo_bin = s.valid ? win.x : found[0];
             A.sel[l] = s;
-            A.cand_count[l] = 0u;
+            if (!s.valid) {
+                A.cand_count[l] = 0u;
+                atomicAdd(&A.status->redo_layers, 1u);
+            }
+            // how far the bin moves from one step to the next is a matter of the layer's size: the k-th largest of a few
+            // thousand values wanders over several bins (an eighth of an octave each), that of millions stays put.  A wide
+            // window costs candidates, so only small layers get one; their second sweep would be cheap anyway.
+            const uint64_t n_l = A.seg_len[l];
+            const uint32_t half = n_l >= (1ull << 19) ? 0u : (n_l >= (1ull << 13) ? 3u : 8u);
+            A.window[l] = make_uint2(found[0] > half ? found[0] - half : 0u, min(found[0] + half, (uint32_t)kHistBins - 1u));
         }
     }
     double s1 = 0.0, s2 = 0.0, sa = 0.0, bad = 0.0;
     uint32_t amax = 0u, amin = 0xFFFFFFFFu;
     // every item summed around its own pivot; here the sums are moved to the pivot of the layer's first item
-    const double pivot = (double)A.p_piv[lo];
+    const float pivot_f = lo < hi ? A.p_piv[lo] : 0.f;
+    const double pivot = (double)pivot_f;
+    double n_local = 0.0;
 #pragma unroll 4
     for (uint32_t i = lo + tid; i < hi; i += kThreads) {
         const MomentSums m = rebase(A.p_s1[i], A.p_s2[i], (double)A.items[i].len, (double)A.p_piv[i], pivot);
         s1 += m.s1;
         s2 += m.s2;
+        n_local += (double)A.items[i].len;
         bad += (double)A.p_bad[i];
         if (A.has_hz) {
             amax = max(amax, A.p_amax[i]);
@@ -749,10 +940,18 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     s2 = block_sum(s2, red);
     sa = block_sum(sa, red);
     bad = block_sum(bad, red);
+    if (A.record_out) n_local = block_sum(n_local, red);
     amax = __reduce_max_sync(0xFFFFFFFFu, amax);
     amin = __reduce_min_sync(0xFFFFFFFFu, amin);
     if ((tid & 31) == 0) { red_u[0][tid >> 5] = amax; red_u[1][tid >> 5] = amin; }
     __syncthreads();
+    if (A.record_out) {
+        if (tid == 0) {
+            for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
+            A.record_out[l] = LayerRecord{s1, s2, n_local, pivot_f, amax, amin, (uint32_t)min(bad, 4294967295.0)};
+        }
+        return;
+    }
     if (tid == 0) {
         for (int w = 1; w < kWarps; ++w) { amax = max(amax, red_u[0][w]); amin = min(amin, red_u[1][w]); }
         const double n = (double)A.seg_len[l];
@@ -771,21 +970,40 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    double total_bad = 0.0;
-    for (uint32_t j = tid; j < A.L; j += kThreads)
-        total_bad += (double)__ldcg(&A.scratch[j].bad);
-    total_bad = block_sum(total_bad, red);
-    double near = 0.0;
-    if (total_bad == 0.0)
-        for (uint32_t j = tid; j < A.L; j += kThreads) near += (double)commit_layer(A, j);
-    near = block_sum(near, red);
-    if (tid == 0) {
-        A.status->step = A.step;
-        A.status->nonfinite = (unsigned long long)total_bad;
-        A.status->skipped = total_bad != 0.0 ? 1u : 0u;
-        if (A.control && total_bad == 0.0) A.status->near_count = (uint32_t)near;
-        A.status->done_counter = 0u;
+    commit_step(A, red);
+}
+
+// Sharded pass: the records of all ranks for every layer, [world][L], combined in rank order (so that every rank
+// arrives at the same numbers), give the layer's statistics.  One thread per layer.
+__global__ void __launch_bounds__(kThreads) k_merge_records(const LayerRecord *all, uint32_t world, uint32_t L, LayerScratch *scratch)
+{
+    const uint32_t l = blockIdx.x * kThreads + threadIdx.x;
+    if (l >= L) return;
+    double pivot = 0.0, s1 = 0.0, s2 = 0.0, n = 0.0, bad = 0.0;
+    uint32_t amax = 0u, amin = 0xFFFFFFFFu;
+    bool have = false;
+    for (uint32_t r = 0; r < world; ++r) {
+        const LayerRecord x = all[(size_t)r * L + l];
+        if (!(x.n > 0.0)) continue;
+        if (!have) { pivot = (double)x.pivot; have = true; }
+        const MomentSums m = rebase(x.s1, x.s2, x.n, (double)x.pivot, pivot);
+        s1 += m.s1; s2 += m.s2; n += x.n; bad += (double)x.bad;
+        amax = max(amax, x.amax); amin = min(amin, x.amin);
     }
+    const double shift = n > 0.0 ? s1 / n : 0.0;
+    double var = n > 0.0 ? s2 / n - shift * shift : 0.0;
+    if (!(var > 0.0)) var = 0.0;
+    LayerScratch sc;
+    sc.mean = pivot + shift; sc.var = var; sc.sum_abs = 0.0;
+    sc.bad = (unsigned long long)bad;
+    sc.amax = amax; sc.amin = amin;
+    scratch[l] = sc;
+}
+
+__global__ void __launch_bounds__(kThreads) k_commit(const DecideArgs A)
+{
+    __shared__ double red[kWarps];
+    commit_step(A, red);
 }
 
 // ------------------------------------------------------------------ phase B: update + cast
@@ -1595,174 +1813,22 @@ __global__ void __launch_bounds__(kThreads) k_probe(float *z, uint64_t n_vec, ui
 
 // ------------------------------------------------------------------ top-k: radix select on |S| bit patterns
 //
-// |S| >= 0, so the order of the values is the order of their 31-bit patterns.  Level 1 (bits 30..20)
-// is counted during the sweep.  k_decide finds, per layer, the bin b1 that holds the k-th largest
-// value.  One more pass over |S| (k_mask_compact) sets the mask bits of every element in a bin above
-// b1 and appends the elements of bin b1 (value, index in layer) to the layer's candidate list.
-// k_resolve then finishes the selection on the candidates alone: two more value digits and, if more
-// candidates equal the threshold than are to be taken, three digits of the index (lower index first).
-// The result does not depend on the order in which candidates were appended.
-
-struct MaskArgs {
-    const Item *items;
-    uint32_t n_items, n_batches;
-    const float *abs_s;
-    uint32_t *mask;
-    double *p_mass;              // per item: sum of |S| in bins above the layer's level-1 bin
-    const SelectState *sel;
-    const uint64_t *seg_off, *seg_len;
-    uint32_t *cand_count;        // [L]
-    uint32_t *cand_val;          // [n_total], candidates of layer l at seg_off[l] ...
-    uint32_t *cand_idx;          // [n_total]
-    const Status *status;
-};
-
-constexpr uint32_t kStageCap = 384;      // candidates a warp collects in shared memory before it reserves list slots
-
-// Stages this lane's candidates (bit e of `cand` = element e of its vector) in the warp's shared-memory
-// buffer, behind the `running` ones already there.  Whole warp; `running` stays warp-uniform.
-__device__ __forceinline__ void stage_candidates(uint32_t cand, const uint32_t (&ab)[4], uint32_t local0, uint32_t lane,
-                                                 uint32_t &running, uint32_t *sval, uint32_t *sidx)
-{
-    if (!__any_sync(0xFFFFFFFFu, cand != 0u)) return;
-    const uint32_t n_mine = (uint32_t)__popc(cand);
-    uint32_t incl = n_mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if ((int)lane >= o) incl += t;
-    }
-    uint32_t base = running + incl - n_mine;
-    running += __shfl_sync(0xFFFFFFFFu, incl, 31);
-#pragma unroll
-    for (uint32_t e = 0; e < 4; ++e)
-        if (cand & (1u << e)) { sval[base] = ab[e]; sidx[base] = local0 + e; ++base; }
-}
-
-// 8 lanes make one 32-bit mask word out of their 4-bit pieces.
-__device__ __forceinline__ uint32_t gather_word(uint32_t nib, uint32_t lane)
-{
-    uint32_t word = nib << ((lane & 7u) * 4u);
-    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
-    word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
-    return word;
-}
-
-__global__ void __launch_bounds__(kThreads) k_mask_compact(const MaskArgs A)
-{
-    if (A.status->skipped) return;
-    __shared__ uint32_t sh_val[kWarps][kStageCap];
-    __shared__ uint32_t sh_idx[kWarps][kStageCap];
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
-        const uint32_t it = batch * kWarps + warp;
-        if (it >= A.n_items) continue;
-        const Item item = A.items[it];
-        if (item.len == 0u) { if (lane == 0) A.p_mass[it] = 0.0; continue; }
-        const uint64_t begin = item.begin, end = begin + item.len;
-        const uint64_t seg_b = A.seg_off[item.seg];
-        const uint32_t b1 = A.sel[item.seg].prefix;
-        uint32_t *sval = sh_val[warp], *sidx = sh_idx[warp];
-        uint32_t staged = 0u;
-        double mass = 0.0;
-        // moves the staged candidates to the layer's list: one slot reservation for all of them
-        auto flush = [&]() {
-            if (staged == 0u) return;
-            uint32_t base = 0;
-            if (lane == 0) base = atomicAdd(A.cand_count + item.seg, staged);
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
-            __syncwarp();
-            for (uint32_t j = lane; j < staged; j += 32) {
-                A.cand_val[seg_b + base + j] = sval[j];
-                A.cand_idx[seg_b + base + j] = sidx[j];
-            }
-            __syncwarp();
-            staged = 0u;
-        };
-
-        // a row that is cut by the first or last element of the layer
-        auto partial_row = [&](uint64_t row) {
-            const uint64_t i0 = row * 128ull + lane * 4u;
-            uint32_t ab[4] = {0u, 0u, 0u, 0u};
-            uint32_t nib = 0u, cand = 0u;
-            for (uint32_t e = 0; e < 4; ++e) {
-                if (i0 + e >= begin && i0 + e < end) {
-                    ab[e] = __float_as_uint(A.abs_s[i0 + e]);
-                    const uint32_t bin = ab[e] >> 20;
-                    if (bin > b1) { nib |= 1u << e; mass += (double)__uint_as_float(ab[e]); }
-                    if (bin == b1) cand |= 1u << e;
-                }
-            }
-            if (staged + 128u > kStageCap) flush();
-            stage_candidates(cand, ab, (uint32_t)(i0 - seg_b), lane, staged, sval, sidx);
-            const uint32_t word = gather_word(nib, lane);
-            if ((lane & 7u) == 0u) {
-                const uint64_t w0 = row * 128ull + (lane >> 3) * 32ull;     // first element of this word
-                uint32_t *dst = A.mask + (w0 >> 5);
-                if (w0 >= begin && w0 + 32u <= end) {
-                    *dst = word;
-                } else if (w0 + 32u > begin && w0 < end) {
-                    // the other bits of this word belong to a neighbouring layer or a gap: replace only ours
-                    const uint32_t lo_bit = begin > w0 ? (uint32_t)(begin - w0) : 0u;
-                    const uint32_t hi_bit = end < w0 + 32u ? (uint32_t)(end - w0) : 32u;     // exclusive
-                    const uint32_t ours = (hi_bit == 32u ? 0xFFFFFFFFu : ((1u << hi_bit) - 1u)) & ~((1u << lo_bit) - 1u);
-                    atomicAnd(dst, ~ours);
-                    if (word) atomicOr(dst, word);
-                }
-            }
-        };
-        // a row entirely inside the item: its four mask words are owned by this warp
-        auto full_row = [&](uint64_t row, const float4 v) {
-            const uint32_t ab[4] = {__float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z), __float_as_uint(v.w)};
-            uint32_t nib = 0u, cand = 0u;
-            float above = 0.f;
-#pragma unroll
-            for (uint32_t e = 0; e < 4; ++e) {
-                const uint32_t bin = ab[e] >> 20;
-                if (bin > b1) { nib |= 1u << e; above += __uint_as_float(ab[e]); }
-                if (bin == b1) cand |= 1u << e;
-            }
-            mass += (double)above;
-            if (staged + 128u > kStageCap) flush();
-            stage_candidates(cand, ab, (uint32_t)(row * 128ull - seg_b) + lane * 4u, lane, staged, sval, sidx);
-            const uint32_t word = gather_word(nib, lane);
-            if ((lane & 7u) == 0u) A.mask[row * 4ull + (lane >> 3)] = word;
-        };
-
-        const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
-        const uint64_t full_lo = (begin + 127) >> 7, full_hi = end >> 7;
-        const bool head_partial = (begin & 127u) != 0u;
-        const bool tail_partial = (end & 127u) != 0u && !(head_partial && row_last == row_first);
-        if (head_partial) partial_row(row_first);
-        if (full_hi > full_lo) {
-            constexpr int U = 8;
-            uint64_t row = full_lo;
-            while (row + U <= full_hi) {
-                float4 v[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) v[u] = __ldcs(reinterpret_cast<const float4 *>(A.abs_s + (row + u) * 128ull + lane * 4u));
-#pragma unroll
-                for (int u = 0; u < U; ++u) full_row(row + u, v[u]);
-                row += U;
-            }
-            while (row < full_hi) {
-                full_row(row, __ldcs(reinterpret_cast<const float4 *>(A.abs_s + row * 128ull + lane * 4u)));
-                ++row;
-            }
-        }
-        if (tail_partial) partial_row(row_last);
-        flush();
-        mass = warp_sum(mass);
-        if (lane == 0) A.p_mass[it] = mass;
-    }
-}
+// |S| >= 0, so the order of the values is the order of their 31-bit patterns.  Level 1 (bits 30..20) is counted
+// during the sweep, which also sets the mask bits of every element above a window of bins around the bin that held
+// the k-th largest value at the last step, and lists the elements inside the window as candidates (value, index in
+// layer).  k_decide finds, per layer, the bin b1 that holds the k-th largest value now, and whether the window
+// contains it; layers where it does not are swept once more with the window [b1, b1].  k_apply_resolve then finishes
+// the selection on the candidates alone: those in bins above b1 are taken, those in b1 go through two more value
+// digits and, if more of them equal the threshold than are to be taken, three digits of the index (lower index
+// first).  The result does not depend on the order in which candidates were listed.
 
 struct ResolveArgs {
     const uint32_t *item_lo;
     const uint64_t *seg_off, *seg_len;
     const uint32_t *cand_count, *cand_val, *cand_idx;
-    uint32_t *mask;
+    uint32_t *cand_count_out;      // cleared for the next step once the layer is resolved
+    uint32_t *mask2;               // the two mask buffers
+    uint64_t mask_words;
     const double *p_mass;
     const LayerScratch *scratch;
     SelectState *sel;
@@ -1784,25 +1850,26 @@ __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32
     __shared__ uint32_t scan[kThreads];
     __shared__ uint32_t found[2];
     __shared__ double red[kWarps];
-    __shared__ unsigned long long acc_u64[2];
+    __shared__ unsigned long long acc_u64;
     const uint32_t tid = threadIdx.x;
     const uint64_t off = A.seg_off[l];
     SelectState s = A.sel[l];
     const uint32_t b1 = s.prefix;
+    uint32_t *mask = A.mask2 + (size_t)A.status->mask_cur * A.mask_words;
 
     auto clear = [&](int bins) { for (int b = tid; b < bins; b += kThreads) h[b] = 0u; __syncthreads(); };
 
     const uint32_t m = A.cand_count[l];
     const uint32_t *cv = A.cand_val + off, *ci = A.cand_idx + off;
 
-    // value digits: bits 19..9, then bits 8..0
+    // value digits of the candidates in bin b1: bits 19..9, then bits 8..0
     clear(kHistBins);
     for (uint32_t j0 = 0; j0 < m; j0 += kThreads * kResolveLoads) {
         uint32_t v[kResolveLoads];
 #pragma unroll
         for (int u = 0; u < kResolveLoads; ++u) { const uint32_t j = j0 + u * kThreads + tid; v[u] = j < m ? __ldg(cv + j) : 0xFFFFFFFFu; }
 #pragma unroll
-        for (int u = 0; u < kResolveLoads; ++u) if (v[u] != 0xFFFFFFFFu) atomicAdd(&h[(v[u] >> 9) & 2047u], 1u);
+        for (int u = 0; u < kResolveLoads; ++u) if ((v[u] >> 20) == b1) atomicAdd(&h[(v[u] >> 9) & 2047u], 1u);
     }
     __syncthreads();
     block_find_bin<true>(h, kHistBins, s.remaining, scan, found);
@@ -1848,9 +1915,11 @@ __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32
         idx_limit = prefix;
     }
 
-    // set the bits of the taken candidates; their sum is exact: all share sign and exponent
-    // (the exponent is part of the level-1 digit), so it is count * 2^e + (sum of mantissas) * 2^(e-23)
-    unsigned long long cnt = 0ull, mant = 0ull;
+    // set the bits of the taken candidates.  Their sum is exact: the window spans a few binary exponents at most
+    // (seventeen bins of an eighth of an octave), so every value is an integer multiple of the smallest exponent's unit,
+    // and the integers are added.
+    const uint32_t e_lo = (s.lo_bin >> 3) & 0xFFu, e_unit = e_lo ? e_lo : 1u;      // exponent field 0 (subnormal) counts as 1
+    unsigned long long units = 0ull;
     for (uint32_t j0 = 0; j0 < m; j0 += kThreads * (kResolveLoads / 2)) {
         uint32_t v[kResolveLoads / 2], ix[kResolveLoads / 2];
 #pragma unroll
@@ -1864,36 +1933,28 @@ __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32
             const uint32_t j = j0 + u * kThreads + tid;
             if (j < m && (v[u] > thr || (v[u] == thr && ix[u] <= idx_limit))) {
                 const uint64_t i = off + ix[u];
-                atomicOr(A.mask + (i >> 5), 1u << (i & 31u));
-                ++cnt;
-                mant += v[u] & 0x007FFFFFu;
+                atomicOr(mask + (i >> 5), 1u << (i & 31u));
+                const uint32_t e = v[u] >> 23;
+                const unsigned long long sig = e ? ((v[u] & 0x007FFFFFu) | 0x00800000u) : (v[u] & 0x007FFFFFu);
+                units += sig << ((e ? e : 1u) - e_unit);
             }
         }
     }
-    if (tid < 2) acc_u64[tid] = 0ull;
+    if (tid == 0) acc_u64 = 0ull;
     __syncthreads();
-    atomicAdd(&acc_u64[0], cnt);
-    atomicAdd(&acc_u64[1], mant);
+    atomicAdd(&acc_u64, units);
     double mass = 0.0;
     for (uint32_t i = A.item_lo[l] + tid; i < A.item_lo[l + 1]; i += kThreads) mass += A.p_mass[i];
     mass = block_sum(mass, red);
     if (tid == 0) {
-        const uint32_t expo = (b1 >> 3) & 0xFFu;                      // level-1 digit = 8 exponent bits + 3 mantissa bits
-        const double unit = expo ? ldexp(1.0, (int)expo - 127 - 23) : ldexp(1.0, -126 - 23);
-        const double cand_sum = expo ? ((double)acc_u64[0] * 8388608.0 + (double)acc_u64[1]) * unit
-                                     : (double)acc_u64[1] * unit;
+        const double cand_sum = (double)acc_u64 * ldexp(1.0, (int)e_unit - 127 - 23);
         const double all = A.scratch[l].sum_abs;
         s.thr_bits = thr; s.take_equal = take_equal; s.surplus = n_equal > take_equal ? 1u : 0u;
         A.sel[l] = s;
         A.state[l].thr = __uint_as_float(thr);
         A.state[l].topk_mass = all > 0.0 ? (mass + cand_sum) / all : 1.0;
+        A.cand_count_out[l] = 0u;          // the list is used up; the next sweep starts a new one
     }
-}
-
-__global__ void __launch_bounds__(kThreads) k_resolve(const ResolveArgs A)
-{
-    if (A.status->skipped) return;
-    resolve_layer(A, blockIdx.x);
 }
 
 // Top-k steps: the update needs nothing from the resolve step, so both run in ONE launch.  The first

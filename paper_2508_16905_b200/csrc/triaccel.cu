@@ -33,7 +33,7 @@ struct DeviceBuffers {
     double *p_s1 = nullptr, *p_s2 = nullptr, *p_sa = nullptr, *p_mass = nullptr;
     float *p_piv = nullptr;
     uint32_t *p_amax = nullptr, *p_amin = nullptr, *p_bad = nullptr;
-    float *abs_s = nullptr;
+    uint2 *window = nullptr;                      // top-k: per layer, the level-1 bins the next sweep collects candidates in
     uint32_t *hist = nullptr;
     ta::SelectState *sel = nullptr;
     uint32_t *mask = nullptr;
@@ -81,6 +81,10 @@ struct ta_handle {
     size_t fused_smem = 0;
     unsigned long long barrier_base = 0;  // barrier arrivals of all fused launches so far
     unsigned long long fused_launches = 0;// fused launches since the arrival counters were last cleared
+    bool sharded = false;                 // this handle holds the flat range [range_lo, range_hi) of a model spread over ranks
+    uint64_t range_lo = 0, range_hi = 0;
+    uint64_t pending_step = 0;            // shard: step of a ta_shard_sweep whose ta_shard_apply has not come yet
+    bool pending = false, pending_has_hz = false;
     bool pipe_ok = false;                 // large dense models with TA_FLAG_INPUTS_FINITE: the layer-pipelined launch
     uint32_t pipe_batches = 0;
     int pipe_per_sm = 0;
@@ -122,7 +126,7 @@ void free_all(DeviceBuffers &d)
 {
     void *ptrs[] = {d.pipe_tasks_sweep, d.pipe_tasks_apply, d.pipe_tasks_hold, d.pipe_batch_lo, d.pipe_bsum, d.pipe_layer_done, d.pipe_layer_ready, d.pipe_ctl,
                     d.warp_head, d.block_head, d.block_layer, d.slot_table, d.part, d.mom, d.pw_part, d.pw_coef, d.pw_norm, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2, d.p_piv,
-                    d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.abs_s, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
+                    d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.window, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
     for (void *p : ptrs)
         if (p) cudaFree(p);
@@ -424,7 +428,8 @@ extern "C" {
 
 const char *ta_last_error(const ta_handle *h) { return h ? h->err : g_create_error; }
 
-int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hparams *hp, ta_handle **out)
+static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hparams *hp, uint64_t range_lo,
+                       uint64_t range_hi, bool sharded, ta_handle **out)
 {
     if (out) *out = nullptr;
     g_create_error[0] = 0;
@@ -451,6 +456,11 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         n_params += table[l].length;
     }
     if (end > n_total) return fail(nullptr, TA_ERR_ARG, "ta_create: a segment reaches beyond n_total");
+    if (sharded) {
+        if (range_lo % 128 || range_hi % 128 || range_lo >= range_hi || range_hi > (n_total + 127) / 128 * 128)
+            return fail(nullptr, TA_ERR_ARG, "ta_create_shard: the range must be non-empty, inside the buffer and cut on multiples of 128 elements");
+        if (hp->topk_ppm < 1000000u) return fail(nullptr, TA_ERR_ARG, "ta_create_shard: the top-k mask is not available on a sharded model");
+    }
 
     ta_handle *h = new (std::nothrow) ta_handle;
     if (!h) return fail(nullptr, TA_ERR_NOMEM, "ta_create: out of host memory");
@@ -483,13 +493,16 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     h->table.assign(table, table + L);
     h->topk = hp->topk_ppm < 1000000u;
     h->mask_words = h->topk ? (n_total + 31) / 32 : 0;
+    h->sharded = sharded;
+    h->range_lo = sharded ? range_lo : 0;
+    h->range_hi = sharded ? range_hi : n_total;
 
     // one-launch path for small dense models: needs a cooperative launch with every block resident
     int fused_per_sm = 0;
     {
         int coop = 0;
         TA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device));
-        if (coop && !(hp->flags & TA_FLAG_NO_ONE_LAUNCH) && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f &&
+        if (coop && !sharded && !(hp->flags & TA_FLAG_NO_ONE_LAUNCH) && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f &&
             n_params <= kFusedMaxParams) {
             const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
             h->fused_ok = true;
@@ -546,7 +559,9 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     }
     for (uint32_t l = 0; l < L && !h->fused_ok; ++l) {
         item_lo[l] = (uint32_t)items.size();
-        const uint64_t b = table[l].offset, e = b + table[l].length;
+        // a shard holds the part of every layer that lies inside its range (possibly nothing)
+        const uint64_t b = std::max<uint64_t>(table[l].offset, h->range_lo), e = std::min<uint64_t>(table[l].offset + table[l].length, h->range_hi);
+        if (e <= b) continue;
         // top-k: a layer of at least one full batch starts on a batch boundary, so that its batches hold one
         // layer only and can count their histogram in shared memory (padding items are empty)
         const uint64_t layer_items = (e - 1) / h->item_elems - b / h->item_elems + 1;
@@ -594,10 +609,14 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     if (h->topk) {
         TA_TRY(dev_alloc(&d.p_sa, h->n_items));
         TA_TRY(dev_alloc(&d.p_mass, h->n_items));
-        TA_TRY(dev_alloc(&d.abs_s, n_total));
+        TA_TRY(dev_alloc(&d.window, L));
+        {
+            std::vector<uint2> none(L, make_uint2(1u, 0u));          // no guess before the first step with curvature
+            TA_TRY(cudaMemcpy(d.window, none.data(), L * sizeof(uint2), cudaMemcpyHostToDevice));
+        }
         TA_TRY(dev_alloc(&d.hist, (size_t)L * ta::kHistBins));
         TA_TRY(dev_alloc(&d.sel, L));
-        TA_TRY(dev_alloc(&d.mask, h->mask_words));
+        TA_TRY(dev_alloc(&d.mask, 2 * h->mask_words));           // the current mask and the one being built
         TA_TRY(dev_alloc(&d.cand_count, L));
         TA_TRY(dev_alloc(&d.cand_val, n_total));
         TA_TRY(dev_alloc(&d.cand_idx, n_total));
@@ -607,7 +626,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
         TA_TRY(cudaMemcpy(d.batch_seg, batch_seg.data(), batch_seg.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
         TA_TRY(cudaMemset(d.hist, 0, (size_t)L * ta::kHistBins * sizeof(uint32_t)));
         TA_TRY(cudaMemset(d.sel, 0, (size_t)L * sizeof(ta::SelectState)));
-        TA_TRY(cudaMemset(d.mask, 0, h->mask_words * sizeof(uint32_t)));
+        TA_TRY(cudaMemset(d.mask, 0, 2 * h->mask_words * sizeof(uint32_t)));
     }
     TA_TRY(cudaMemcpy(d.items, items.data(), items.size() * sizeof(ta::Item), cudaMemcpyHostToDevice));
     TA_TRY(cudaMemcpy(d.item_lo, item_lo.data(), (L + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice));
@@ -626,6 +645,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
     TA_TRY(cudaMemset(d.scratch, 0, L * sizeof(ta::LayerScratch)));
     TA_TRY(cudaMemset(d.status, 0, sizeof(ta::Status)));
     if (hp->momentum != 0.f) {
+        if (sharded) { snprintf(h->err, 256, "ta_create_shard: momentum is not available on a sharded model"); return bail(TA_ERR_ARG); }
         TA_TRY(dev_alloc(&d.mom, n_total));
         TA_TRY(cudaMemset(d.mom, 0, n_total * sizeof(float)));
     }
@@ -653,7 +673,7 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
             }
         }
     }
-    if ((hp->flags & TA_FLAG_INPUTS_FINITE) && !h->fused_ok && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f) {
+    if ((hp->flags & TA_FLAG_INPUTS_FINITE) && !sharded && !h->fused_ok && !h->topk && hp->momentum == 0.f && hp->weight_decay == 0.f) {
         // the layer-pipelined launch: its own (finer) items, the two task queues and the per-layer counters
         const PipePlan pl = plan_pipe(table, L);
         if (L < (1u << 30) && pl.sweep.size() < 0xFFFFFFFFull) {
@@ -691,6 +711,17 @@ int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hp
 #undef TA_TRY
     *out = h;
     return TA_OK;
+}
+
+int ta_create(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hparams *hp, ta_handle **out)
+{
+    return create_impl(table, L, n_total, hp, 0, n_total, false, out);
+}
+
+int ta_create_shard(const ta_segment *table, uint32_t L, uint64_t n_total, const ta_hparams *hp, uint64_t range_lo,
+                    uint64_t range_hi, ta_handle **out)
+{
+    return create_impl(table, L, n_total, hp, range_lo, range_hi, true, out);
 }
 
 int ta_destroy(ta_handle *h)
@@ -822,6 +853,7 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
         return fail(h, TA_ERR_ALIGN, "ta_step: every device pointer must be 16-byte aligned");
     if (step >= (1ull << 32)) return fail(h, TA_ERR_ARG, "ta_step: step must be below 2^32");
     if (h->stepped && step <= h->last_step) return fail(h, TA_ERR_STATE, "ta_step: step must increase from call to call");
+    if (h->sharded) return fail(h, TA_ERR_STATE, "ta_step: this handle holds a shard; use ta_shard_sweep and ta_shard_apply");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool bf16 = h->hp.grad_dtype == TA_GRAD_BF16;
     const int P = Hz ? (int)h->hp.num_probes : 0;
@@ -896,7 +928,11 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
     sa.g = g; sa.hz = Hz; sa.n_total = h->n_total; sa.seed = probe_seed; sa.step = (uint32_t)step;
     sa.p_s1 = d.p_s1; sa.p_s2 = d.p_s2; sa.p_sa = d.p_sa; sa.p_piv = d.p_piv;
     sa.p_amax = d.p_amax; sa.p_amin = d.p_amin; sa.p_bad = d.p_bad;
-    sa.abs_s = d.abs_s; sa.hist = d.hist; sa.batch_seg = d.batch_seg;
+    sa.hist = d.hist; sa.batch_seg = d.batch_seg;
+    sa.mask2 = d.mask; sa.mask_words = h->mask_words; sa.window = d.window; sa.sel = d.sel;
+    sa.cand_count = d.cand_count; sa.cand_val = d.cand_val; sa.cand_idx = d.cand_idx; sa.seg_off = d.seg_off;
+    sa.p_mass = d.p_mass; sa.status = d.status; sa.redo = 0u;
+    if (topk) TA_CUDA(h, cudaMemsetAsync(&d.status->redo_layers, 0, sizeof(uint32_t), s));
     const bool ok = bf16 ? dispatch_sweep<true>(h, P, sa, s) : dispatch_sweep<false>(h, P, sa, s);
     if (!ok) return fail(h, TA_ERR_ARG, "ta_step: unsupported probe count");
     if (timed) cudaEventRecord(ev[1], s);
@@ -909,38 +945,34 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
     da.hp = hyper_of(h->hp); da.eta0 = h->hp.eta0; da.L = h->L;
     da.has_hz = Hz ? 1u : 0u; da.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; da.topk = topk ? 1u : 0u;
     da.step = step;
-    da.hist = d.hist; da.sel = d.sel; da.cand_count = d.cand_count; da.seg_k = d.seg_k;
+    da.hist = d.hist; da.sel = d.sel; da.cand_count = d.cand_count; da.seg_k = d.seg_k; da.window = d.window;
     ta::k_decide<<<h->L, ta::kThreads, 0, s>>>(da);
     ++h->launches;
 
     if (topk) {
+        // layers whose selection window missed are swept once more with the exact bin (nothing to do in the common case)
+        sa.redo = 1u;
+        if (!(bf16 ? dispatch_sweep<true>(h, P, sa, s) : dispatch_sweep<false>(h, P, sa, s)))
+            return fail(h, TA_ERR_ARG, "ta_step: unsupported probe count");
         const int grid = grid_for(h);
-        ta::MaskArgs ma{d.items, h->n_items, h->n_batches, d.abs_s, d.mask, d.p_mass, d.sel, d.seg_off, d.seg_len,
-                        d.cand_count, d.cand_val, d.cand_idx, d.status};
-        ta::k_mask_compact<<<grid, ta::kThreads, 0, s>>>(ma);
-        ta::ResolveArgs ra{d.item_lo, d.seg_off, d.seg_len, d.cand_count, d.cand_val, d.cand_idx, d.mask, d.p_mass,
-                           d.scratch, d.sel, d.state, d.status};
-        // the update needs nothing from the resolve step: both run in one launch (k_apply_resolve) unless the
-        // caller applies the update itself
-        if (!defer_apply) {
-            if (timed) cudaEventRecord(ev[2], s);
-            ta::ApplyArgs aa{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status, d.mom, h->hp.momentum, h->hp.weight_decay};
-            const unsigned blocks = (unsigned)h->L + (unsigned)grid;
-            const bool mom = d.mom != nullptr;
-            if (bf16 && mom) ta::k_apply_resolve<true, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-            else if (bf16) ta::k_apply_resolve<true, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-            else if (mom) ta::k_apply_resolve<false, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-            else ta::k_apply_resolve<false, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-            h->launches += 2;
-            if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
-            TA_CUDA(h, cudaGetLastError());
-            h->stepped = true;
-            h->last_step = step;
-            h->last_stream = s;
-            return TA_OK;
-        }
-        ta::k_resolve<<<h->L, ta::kThreads, 0, s>>>(ra);
-        h->launches += 2;
+        ta::ResolveArgs ra{d.item_lo, d.seg_off, d.seg_len, d.cand_count, d.cand_val, d.cand_idx, d.cand_count, d.mask,
+                           h->mask_words, d.p_mass, d.scratch, d.sel, d.state, d.status};
+        // the update needs nothing from the resolve step: both run in one launch (k_apply_resolve)
+        if (timed) cudaEventRecord(ev[2], s);
+        ta::ApplyArgs aa{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status, d.mom, h->hp.momentum, h->hp.weight_decay};
+        const unsigned blocks = (unsigned)h->L + (unsigned)grid;
+        const bool mom = d.mom != nullptr;
+        if (bf16 && mom) ta::k_apply_resolve<true, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+        else if (bf16) ta::k_apply_resolve<true, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+        else if (mom) ta::k_apply_resolve<false, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+        else ta::k_apply_resolve<false, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+        ++h->launches;
+        if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
+        TA_CUDA(h, cudaGetLastError());
+        h->stepped = true;
+        h->last_step = step;
+        h->last_stream = s;
+        return TA_OK;
     }
 
     if (timed) cudaEventRecord(ev[2], s);
@@ -1060,6 +1092,81 @@ int ta_step_host(ta_handle *h, float *w_host, const void *g_host, const float *H
     return TA_OK;
 }
 
+int ta_shard_sweep(ta_handle *h, const void *g_local, const float *Hz_local, uint64_t probe_seed, uint64_t step,
+                   ta_layer_record *records_out, void *stream)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!h->sharded) return fail(h, TA_ERR_STATE, "ta_shard_sweep: the handle was not made by ta_create_shard");
+    if (!g_local || !records_out) return fail(h, TA_ERR_ARG, "ta_shard_sweep: g and records_out must not be NULL");
+    if (!aligned16(g_local) || !aligned16(Hz_local) || (reinterpret_cast<uintptr_t>(records_out) & 7u))
+        return fail(h, TA_ERR_ALIGN, "ta_shard_sweep: g and Hz must be 16-byte aligned, records_out 8-byte aligned");
+    if (step >= (1ull << 32)) return fail(h, TA_ERR_ARG, "ta_shard_sweep: step must be below 2^32");
+    if (h->stepped && step <= h->last_step) return fail(h, TA_ERR_STATE, "ta_shard_sweep: step must increase from call to call");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DeviceBuffers &d = h->d;
+    const bool bf16 = h->hp.grad_dtype == TA_GRAD_BF16;
+    const int P = Hz_local ? (int)h->hp.num_probes : 0;
+    const uint64_t local_n = h->range_hi - h->range_lo;
+    // the kernels index by flat element (the probes depend on it): the local buffers are addressed through bases moved
+    // back by the start of the range; only elements inside the range are ever touched
+    ta::SweepArgs sa{};
+    sa.items = d.items; sa.n_items = h->n_items; sa.n_batches = h->n_batches;
+    sa.g = static_cast<const char *>(g_local) - h->range_lo * (bf16 ? 2 : 4);
+    sa.hz = Hz_local ? Hz_local - h->range_lo : nullptr;
+    sa.n_total = local_n; sa.seed = probe_seed; sa.step = (uint32_t)step;
+    sa.p_s1 = d.p_s1; sa.p_s2 = d.p_s2; sa.p_sa = d.p_sa; sa.p_piv = d.p_piv;
+    sa.p_amax = d.p_amax; sa.p_amin = d.p_amin; sa.p_bad = d.p_bad;
+    if (h->n_items) {
+        if (!(bf16 ? dispatch_sweep<true>(h, P, sa, s) : dispatch_sweep<false>(h, P, sa, s)))
+            return fail(h, TA_ERR_ARG, "ta_shard_sweep: unsupported probe count");
+    }
+    ta::DecideArgs da{};
+    da.item_lo = d.item_lo; da.seg_len = d.seg_len; da.items = d.items;
+    da.p_s1 = d.p_s1; da.p_s2 = d.p_s2; da.p_sa = d.p_sa; da.p_piv = d.p_piv;
+    da.p_amax = d.p_amax; da.p_amin = d.p_amin; da.p_bad = d.p_bad;
+    da.has_hz = Hz_local ? 1u : 0u; da.L = h->L;
+    da.record_out = reinterpret_cast<ta::LayerRecord *>(records_out);
+    ta::k_decide<<<h->L, ta::kThreads, 0, s>>>(da);
+    ++h->launches;
+    TA_CUDA(h, cudaGetLastError());
+    h->pending_step = step;
+    h->pending = true;
+    h->pending_has_hz = Hz_local != nullptr;
+    h->last_stream = s;
+    return TA_OK;
+}
+
+int ta_shard_apply(ta_handle *h, float *w_local, const void *g_local, uint16_t *c_local, const ta_layer_record *records_all,
+                   uint32_t world, void *stream)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!h->sharded) return fail(h, TA_ERR_STATE, "ta_shard_apply: the handle was not made by ta_create_shard");
+    if (!w_local || !g_local || !c_local || !records_all || world == 0) return fail(h, TA_ERR_ARG, "ta_shard_apply: NULL argument");
+    if (!aligned16(w_local) || !aligned16(g_local) || !aligned16(c_local) || (reinterpret_cast<uintptr_t>(records_all) & 7u))
+        return fail(h, TA_ERR_ALIGN, "ta_shard_apply: w, g and c must be 16-byte aligned, records_all 8-byte aligned");
+    if (!h->pending) return fail(h, TA_ERR_STATE, "ta_shard_apply: no ta_shard_sweep is waiting for its records");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DeviceBuffers &d = h->d;
+    const bool bf16 = h->hp.grad_dtype == TA_GRAD_BF16;
+    const uint64_t step = h->pending_step;
+    ta::k_merge_records<<<(h->L + ta::kThreads - 1) / ta::kThreads, ta::kThreads, 0, s>>>(
+        reinterpret_cast<const ta::LayerRecord *>(records_all), world, h->L, d.scratch);
+    ta::DecideArgs da{};
+    da.scratch = d.scratch; da.state = d.state; da.status = d.status;
+    da.hp = hyper_of(h->hp); da.eta0 = h->hp.eta0; da.L = h->L;
+    da.has_hz = h->pending_has_hz ? 1u : 0u; da.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; da.topk = 0u;
+    da.step = step;
+    ta::k_commit<<<1, ta::kThreads, 0, s>>>(da);
+    h->launches += 2;
+    launch_apply(h, w_local - h->range_lo, static_cast<const char *>(g_local) - h->range_lo * (bf16 ? 2 : 4), c_local - h->range_lo, 0, h->n_items, s);
+    TA_CUDA(h, cudaGetLastError());
+    h->stepped = true;
+    h->last_step = step;
+    h->pending = false;
+    h->last_stream = s;
+    return TA_OK;
+}
+
 int ta_power_iterate(ta_handle *h, const float *u, const float *Hu, const float *V, const float *lambda_V, uint32_t m,
                      float *u_next, float *lambda_out, float *norm_out, void *stream)
 {
@@ -1174,8 +1281,14 @@ int ta_precision_codes(ta_handle *h, uint8_t *out_host)
 int ta_masks(ta_handle *h, const uint32_t **dev_bits, uint64_t *num_words)
 {
     if (!h || !dev_bits || !num_words) return TA_ERR_ARG;
-    *dev_bits = h->topk ? h->d.mask : nullptr;
+    *dev_bits = nullptr;
     *num_words = h->mask_words;
+    if (!h->topk) return TA_OK;
+    // two buffers take turns; which one holds the mask is decided on the device when a step commits
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    ta::Status st;
+    TA_CUDA(h, cudaMemcpy(&st, h->d.status, sizeof(st), cudaMemcpyDeviceToHost));
+    *dev_bits = h->d.mask + (size_t)(st.mask_cur & 1u) * h->mask_words;
     return TA_OK;
 }
 
@@ -1203,8 +1316,9 @@ int ta_state_save(ta_handle *h, void *buf_host, uint64_t bytes)
     TA_CUDA(h, cudaMemcpy(p, h->d.state, h->L * sizeof(ta::LayerState), cudaMemcpyDeviceToHost));
     p += h->L * sizeof(ta::LayerState);
     TA_CUDA(h, cudaMemcpy(p, h->d.status, sizeof(ta::Status), cudaMemcpyDeviceToHost));
+    const uint32_t mask_cur = reinterpret_cast<const ta::Status *>(p)->mask_cur & 1u;
     p += sizeof(ta::Status);
-    if (h->mask_words) TA_CUDA(h, cudaMemcpy(p, h->d.mask, h->mask_words * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (h->mask_words) TA_CUDA(h, cudaMemcpy(p, h->d.mask + (size_t)mask_cur * h->mask_words, h->mask_words * sizeof(uint32_t), cudaMemcpyDeviceToHost));
     p += h->mask_words * sizeof(uint32_t);
     if (h->d.mom) TA_CUDA(h, cudaMemcpy(p, h->d.mom, h->n_total * sizeof(float), cudaMemcpyDeviceToHost));
     return TA_OK;
@@ -1229,8 +1343,10 @@ int ta_state_load(ta_handle *h, const void *buf_host, uint64_t bytes)
     TA_CUDA(h, cudaMemcpy(h->d.state, p, h->L * sizeof(ta::LayerState), cudaMemcpyHostToDevice));
     p += h->L * sizeof(ta::LayerState);
     TA_CUDA(h, cudaMemcpy(h->d.status, p, sizeof(ta::Status), cudaMemcpyHostToDevice));
+    ta::Status loaded;
+    std::memcpy(&loaded, p, sizeof(loaded));
     p += sizeof(ta::Status);
-    if (h->mask_words) TA_CUDA(h, cudaMemcpy(h->d.mask, p, h->mask_words * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    if (h->mask_words) TA_CUDA(h, cudaMemcpy(h->d.mask + (size_t)(loaded.mask_cur & 1u) * h->mask_words, p, h->mask_words * sizeof(uint32_t), cudaMemcpyHostToDevice));
     p += h->mask_words * sizeof(uint32_t);
     if (h->d.mom) TA_CUDA(h, cudaMemcpy(h->d.mom, p, h->n_total * sizeof(float), cudaMemcpyHostToDevice));
     h->hp.eta0 = hd.hp.eta0;

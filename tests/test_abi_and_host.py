@@ -11,7 +11,7 @@ import pytest
 import torch
 
 import paper_2508_16905_b200 as ta
-from paper_2508_16905_b200 import binding, workloads as W
+from paper_2508_16905_b200 import binding, dist as D_mod, workloads as W
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -189,6 +189,40 @@ print("rank", rank, "ok")
     path.write_text(script)
     res = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
                           "--master-addr", "127.0.0.1", "--master-port", "29571", str(path)],
+                         capture_output=True, text=True, env=env, timeout=240)
+    assert res.returncode == 0, res.stderr[-2000:]
+    assert res.stdout.count("ok") == 2
+
+
+def test_shard_ranges_and_record_exchange_world_size_2_gloo(tmp_path):
+    # the ranges tile the buffer on the 128-element grid; the exchange returns every rank's records in rank order,
+    # identical on all ranks (which is what makes every rank take the same decisions)
+    for n_total, world in [(4096, 2), (1000, 3), (1311080448, 8), (128, 4)]:
+        r = D_mod.shard_ranges(n_total, world)
+        assert r[0][0] == 0 and r[-1][1] >= n_total and all(a % 128 == 0 and b % 128 == 0 and a <= b for a, b in r)
+        assert all(r[i][1] == r[i + 1][0] for i in range(world - 1))
+    script = r"""
+import os, sys
+sys.path.insert(0, %r)
+import torch
+from paper_2508_16905_b200 import dist as D
+rank, local_rank, world = D.init("gloo")
+L = 5
+mine = torch.full((L * 40,), rank + 1, dtype=torch.uint8)
+mine[::40] = torch.arange(L, dtype=torch.uint8) + 10 * (rank + 1)
+out = D.gather_records(mine)
+assert out.numel() == world * L * 40
+for r in range(world):
+    part = out[r * L * 40:(r + 1) * L * 40]
+    assert torch.equal(part[::40], torch.arange(L, dtype=torch.uint8) + 10 * (r + 1)) and int(part[1]) == r + 1
+D.shutdown()
+print("rank", rank, "ok")
+""" % ROOT
+    path = tmp_path / "ranks.py"
+    path.write_text(script)
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
+    res = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                          "--master-addr", "127.0.0.1", "--master-port", "29573", str(path)],
                          capture_output=True, text=True, env=env, timeout=240)
     assert res.returncode == 0, res.stderr[-2000:]
     assert res.stdout.count("ok") == 2

@@ -162,6 +162,29 @@ def test_tie_breaks_lower_index_first():
     assert np.array_equal(bits, (np.arange(70000) < 17500).astype(np.uint32))
 
 
+@pytest.mark.parametrize("P", [1, 4])
+def test_topk_selection_window_hits_drifts_and_misses(P):
+    # the sweep selects inside a window of bins around the bin that held the k-th largest |S| at the last curvature
+    # step; the curvature of the layers stays, drifts by a few per cent (inside the window), jumps up and down by
+    # large factors (outside: the layer is swept again), and some steps bring no curvature at all
+    table, n_total = ragged_table([70000, 5000, 129, 300000, 33, 2048])
+    rng = np.random.default_rng(21 + P)
+    hp = dict(topk_ppm=100000, num_probes=P, tau_curv=0.5, alpha=2.0, eta0=0.05)
+    run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
+    D0 = np.exp(rng.uniform(np.log(1e-4), 0.0, n_total)).astype(np.float32)
+    factors = [1.0, 1.0, 1.04, 16.0, None, 16.0, 0.01, 0.0104, 1.0]
+    for t, f in enumerate(factors, start=1):
+        g = torch.from_numpy((rng.standard_normal(n_total) * 1e-3).astype(np.float32)).cuda()
+        hz = None
+        if f is not None:
+            D = D0 * np.float32(f)
+            if t == 6:
+                D[table[3][0]:table[3][0] + 300000] = D0[table[3][0]:table[3][0] + 300000]      # one layer stays where it was
+            hz = oracle_hz(D, P, 3, t)
+        run.step(t, g, hz, 3)
+    assert ta.ta_launch_count(run.h) == 4 * 8 + 3          # sweep, decisions, second sweep, resolve + update; 3 kernels without curvature
+
+
 def test_zero_gradient_step_is_identity():
     wl = W.get("mlp_tiny")
     w0 = W.make_weights(wl, "cuda")
