@@ -25,7 +25,8 @@
  *   - There is no CPU fallback: without a usable CUDA device ta_create fails with TA_ERR_CUDA.
  *   - Flat-buffer layout: element i of layer l lives at flat index offset_l + i.  All flat
  *     buffers (w, g, c, each probe of Hz, z_out) have n_total elements and use the same index.
- *     Elements outside every segment ("gaps") are never read or written.
+ *     Elements outside every segment ("gaps") are never used or written (a 16-byte vector that straddles the
+ *     edge of a segment may be fetched whole; the elements outside are masked out).
  */
 #ifndef TRIACCEL_H
 #define TRIACCEL_H

@@ -178,6 +178,20 @@ __device__ __forceinline__ uint2 ld_no_l1(const uint2 *p)
     return v;
 }
 
+// Asynchronous copies to shared memory (no register is held while the data travels).
+__device__ __forceinline__ void cp_async16_stream(void *smem, const void *gmem)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async8_stream(void *smem, const void *gmem)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit_group() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 template <bool BF16> struct GradVec;
 template <> struct GradVec<false> {
     static __device__ __forceinline__ float4 load4(const void *g, uint64_t i, bool stream)
@@ -422,14 +436,19 @@ struct ItemSums {
 // One batch (eight items, one per warp) of the sweep.  Called by the whole block.  `store(it, sums)` is called by
 // lane 0 of each warp with the results of item `it`.  APPLY: the single-pass variant, which also updates the weights
 // of the rows it sweeps (with the step size and code the layers had before this step) and writes their 16-bit copies.
-template <int P, bool BF16, bool TOPK, bool APPLY, int ROWS = 0, typename Store>
+// RING > 0: full rows travel through a ring of RING rows per warp in shared memory (sh_ring, [kWarps][RING][1 + P] rows
+// of 32 x 16 bytes), filled by asynchronous copies that run ahead of the arithmetic: a warp then has loads in flight
+// all the time, not only between two bursts, which is what the multi-probe sweeps (many instructions per byte) need.
+template <int P, bool BF16, bool TOPK, bool APPLY, int ROWS = 0, int RING = 0, typename Store>
 __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, uint32_t *sh_hist, const Store &store,
                                             const SinglePass &sp = SinglePass{nullptr, nullptr, nullptr, 0.f},
-                                            uint32_t *sh_stage = nullptr /* TOPK: [kWarps][2][kStageCap] */)
+                                            uint32_t *sh_stage = nullptr /* TOPK: [kWarps][2][kStageCap] */,
+                                            float4 *sh_ring = nullptr)
 {
+    static_assert(!(RING > 0 && (APPLY || P == 0)), "the ring is for sweeps with probe products");
     static_assert(!(APPLY && TOPK), "the single-pass variant is for dense curvature");
     constexpr int PP = P > 0 ? P : 1;
-    constexpr int U = ROWS > 0 ? ROWS : (P <= 1) ? (BF16 ? TA_SWEEP_ROWS_P1_BF16 : TA_SWEEP_ROWS_P1)
+    constexpr int U = RING > 0 ? 1 : ROWS > 0 ? ROWS : (P <= 1) ? (BF16 ? TA_SWEEP_ROWS_P1_BF16 : TA_SWEEP_ROWS_P1)
                                : (P == 2 ? TA_SWEEP_ROWS_P2 : TA_SWEEP_ROWS_P4);     // rows in flight per lane
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     {
@@ -638,7 +657,46 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
         const bool head_partial = (begin & 127u) != 0u;
         const bool tail_partial = (end & 127u) != 0u && !(head_partial && row_last == row_first);
         if (head_partial) partial_row(row_first);
-        if (full_hi > full_lo) {
+        if constexpr (RING > 0) {
+            if (full_hi > full_lo) {
+            // this lane's 16-byte pieces of RING rows are on their way while it works on the oldest one; a lane reads
+            // back only what it copied itself, so the wait for its own copies is all the ordering needed
+            float4 *mine = sh_ring + (size_t)warp * RING * (1 + PP) * 32u + lane;
+            auto issue = [&](uint64_t row, int slot) {
+                if (row < full_hi) {
+                    const uint64_t i0 = row * 128ull + lane * 4u;
+                    float4 *dst = mine + (size_t)slot * (1 + PP) * 32u;
+                    if (BF16) cp_async8_stream(dst, static_cast<const uint16_t *>(A.g) + i0);
+                    else cp_async16_stream(dst, static_cast<const float *>(A.g) + i0);
+#pragma unroll
+                    for (int p = 0; p < PP; ++p) cp_async16_stream(dst + (size_t)(1 + p) * 32u, A.hz + (uint64_t)p * A.n_total + i0);
+                }
+                cp_async_commit_group();          // one group per row, empty behind the last row, so that the count below holds
+            };
+#pragma unroll
+            for (int r = 0; r < RING; ++r) issue(full_lo + r, r);
+            int slot = 0;
+            for (uint64_t row = full_lo; row < full_hi; ++row) {
+                cp_async_wait_group<RING - 1>();
+                refresh(row);
+                const float4 *src = mine + (size_t)slot * (1 + PP) * 32u;
+                RowData<P> rd[1];
+                if (BF16) {
+                    const uint2 v = *reinterpret_cast<const uint2 *>(src);
+                    rd[0].g = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
+                                          __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+                } else {
+                    rd[0].g = src[0];
+                }
+#pragma unroll
+                for (int p = 0; p < PP; ++p) rd[0].hz[p] = src[(size_t)(1 + p) * 32u];
+                issue(row + RING, slot);          // the slot is free again: the values are in registers
+                full_rows(row, rd, 1);
+                slot = slot + 1 == RING ? 0 : slot + 1;
+            }
+            cp_async_wait_group<0>();
+            }
+        } else if (full_hi > full_lo) {
             uint64_t row = full_lo;
             RowData<P> rd[U];
             // single rows up to the next multiple of U, so that an unrolled group never crosses a 32-row block
@@ -701,11 +759,17 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
     }
 }
 
+// Rows per warp in the shared-memory ring of the top-k sweeps: two blocks per SM must fit with their 32 KB of
+// histogram and candidate staging (3 rows of 2.5 KB with four probes: 61 KB per block).
+__host__ __device__ constexpr int sweep_ring_rows(int P) { return P >= 8 ? 2 : (P >= 4 ? 3 : (P == 2 ? 4 : 6)); }
+__host__ __device__ constexpr size_t sweep_ring_bytes(int P) { return (size_t)kWarps * sweep_ring_rows(P) * (1 + P) * 512u; }
+
 template <int P, bool BF16, bool TOPK>
-__global__ void __launch_bounds__(kThreads, (P == 4 ? TA_SWEEP_MIN_BLOCKS_P4 : 1)) k_sweep(const SweepArgs A)
+__global__ void __launch_bounds__(kThreads, ((P == 4 || TOPK) && P <= 4 ? 2 : 1)) k_sweep(const SweepArgs A)
 {
     __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
     __shared__ uint32_t sh_stage[TOPK ? kWarps * 2 * kStageCap : 1];
+    extern __shared__ __align__(16) float4 sh_ring[];          // TOPK: kWarps * kSweepRing<P> rows of (1 + P) x 512 bytes
     if (TOPK && A.redo && (A.status->skipped || A.status->redo_layers == 0u)) return;      // nothing to repeat
     auto store = [&A](uint32_t it, const ItemSums &r) {
         A.p_s1[it] = r.s1;
@@ -715,7 +779,7 @@ __global__ void __launch_bounds__(kThreads, (P == 4 ? TA_SWEEP_MIN_BLOCKS_P4 : 1
         if (P > 0) { A.p_amax[it] = r.amax; A.p_amin[it] = r.amin; }
         if (TOPK) A.p_sa[it] = r.sa;
     };
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK, false>(A, batch, sh_hist, store, SinglePass{nullptr, nullptr, nullptr, 0.f}, sh_stage);
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK, false, 0, (TOPK ? sweep_ring_rows(P) : 0)>(A, batch, sh_hist, store, SinglePass{nullptr, nullptr, nullptr, 0.f}, sh_stage, sh_ring);
 }
 
 // ------------------------------------------------------------------ decisions

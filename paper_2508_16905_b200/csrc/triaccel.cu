@@ -162,7 +162,16 @@ ta::Hyper hyper_of(const ta_hparams &hp)
 
 template <int P, bool BF16, bool TOPK> void launch_sweep(ta_handle *h, const ta::SweepArgs &a, cudaStream_t s)
 {
-    ta::k_sweep<P, BF16, TOPK><<<grid_for(h), ta::kThreads, 0, s>>>(a);
+    // the top-k sweeps stage their rows in a ring of shared memory (beyond the 48 KB a launch gets without asking)
+    const size_t ring = TOPK ? ta::sweep_ring_bytes(P) : 0;
+    if (TOPK) {
+        static bool asked = false;          // per instantiation
+        if (!asked) {
+            cudaFuncSetAttribute(ta::k_sweep<P, BF16, TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring);
+            asked = true;
+        }
+    }
+    ta::k_sweep<P, BF16, TOPK><<<grid_for(h), ta::kThreads, ring, s>>>(a);
     ++h->launches;
 }
 
