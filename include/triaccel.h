@@ -106,6 +106,13 @@ typedef struct {
  * kernels on small tables.
  */
 #define TA_FLAG_NO_ONE_LAUNCH 2u
+/*
+ * TA_FLAG_GUARD_WORKSPACES -- a test aid: every device buffer that ta_create allocates for the handle (plans, per-item
+ * and per-layer sums, candidate lists, masks, counters) gets 256 guard bytes on either side, and
+ * ta_test_check_guards() tells whether any kernel of the pass has written there (TA_ERR_STATE, with the buffer's
+ * number in ta_last_error).  Results and speed of the pass are unchanged.
+ */
+#define TA_FLAG_GUARD_WORKSPACES 4u
 
 /* Per-layer statistics as of the last ta_step (host side, filled by ta_stats). */
 typedef struct {
@@ -301,6 +308,8 @@ int ta_timing_end(ta_handle *h, double *ms_sweep, double *ms_decide, double *ms_
  * exercised without hanging or faulting the GPU.  TA_ERR_STATE if the handle does not use that path.
  */
 int ta_test_expire_next_wait(ta_handle *h);
+/* Waits for the stream, then checks the guard bytes around the handle's workspaces (see TA_FLAG_GUARD_WORKSPACES). */
+int ta_test_check_guards(ta_handle *h);
 
 /*
  * The work plan of the one-launch path, for inspection (host only, no GPU needed).  Small dense models

@@ -16,14 +16,14 @@ LIB_PATH = os.path.join(HERE, "libtriaccel.so")
 TA_OK, TA_ERR_ARG, TA_ERR_ALIGN, TA_ERR_STATE, TA_ERR_CUDA, TA_ERR_NOMEM = 0, -1, -2, -3, -4, -5
 TA_CODE_FP16, TA_CODE_BF16, TA_CODE_FP32 = 0, 1, 2
 TA_GRAD_F32, TA_GRAD_BF16 = 0, 1
-TA_FLAG_INPUTS_FINITE, TA_FLAG_NO_ONE_LAUNCH = 1, 2
+TA_FLAG_INPUTS_FINITE, TA_FLAG_NO_ONE_LAUNCH, TA_FLAG_GUARD_WORKSPACES = 1, 2, 4
 
 EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "ta_probe", "ta_stats",
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
            "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
            "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait",
            "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch", "ta_plan_pipeline",
-           "ta_create_shard", "ta_shard_sweep", "ta_shard_apply"]
+           "ta_create_shard", "ta_shard_sweep", "ta_shard_apply", "ta_test_check_guards"]
 
 
 class ta_segment(C.Structure):
@@ -106,6 +106,7 @@ def lib():
     L.ta_timing_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(u32)]
     L.ta_grad_moments_static.argtypes = [C.POINTER(ta_segment), u32, vp, u32, vp, vp, vp]
     L.ta_test_expire_next_wait.argtypes = [vp]
+    L.ta_test_check_guards.argtypes = [vp]
     L.ta_power_iterate.argtypes = [vp, vp, vp, vp, vp, u32, vp, vp, vp, vp]
     L.ta_set_curvature.argtypes = [vp, vp]
     L.ta_plan_one_launch.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_run), u32, C.POINTER(u32), C.POINTER(u32),
@@ -344,6 +345,10 @@ def ta_plan_pipeline(table, with_decisions=True):
     if rc != TA_OK:
         raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
     return [(t.kind, t.layer, t.begin, t.length) for t in out[:n.value]]
+
+
+def ta_test_check_guards(h):
+    _check(lib().ta_test_check_guards(h.ptr), h.ptr)
 
 
 def ta_test_expire_next_wait(h):

@@ -1179,7 +1179,9 @@ __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
     if (A.status->skipped) return;
     const LayerState *state = A.state;
     auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) apply_batch<BF16, MOM, TA_APPLY_STREAM_W_STORE != 0>(A, batch, decision);
+    // from the end of the buffer to its start: the gradient rows the sweep read last are the ones still in L2
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x)
+        apply_batch<BF16, MOM, TA_APPLY_STREAM_W_STORE != 0>(A, A.n_batches - 1u - batch, decision);
 }
 
 // ------------------------------------------------------------------ one launch for small models

@@ -17,6 +17,11 @@ namespace {
 
 thread_local char g_create_error[256] = "";
 
+struct GuardRec {          // a buffer allocated between guard words: what cudaMalloc returned, what the library uses, its size
+    void *raw, *user;
+    size_t bytes;
+};
+
 struct DeviceBuffers {
     ta::Item *items = nullptr;
     uint32_t *item_lo = nullptr;
@@ -90,6 +95,7 @@ struct ta_handle {
     int pipe_per_sm = 0;
     unsigned long long pipe_base_s = 0, pipe_base_a = 0;
     uint32_t pipe_launches = 0;
+    std::vector<GuardRec> guards;         // TA_FLAG_GUARD_WORKSPACES: the buffers allocated by ta_create, with their guard words
     std::vector<ta::Item> items_host;     // the plan, kept for the pipelined host path
     cudaStream_t copy_back = nullptr;     // ta_step_host: device-to-host copies run beside the host-to-device ones
     std::vector<cudaEvent_t> chunk_done;
@@ -117,19 +123,39 @@ int fail(ta_handle *h, int code, const char *fmt, const char *detail = "")
         }                                                                         \
     } while (0)
 
+// A library-owned buffer allocated with guard words on both sides (TA_FLAG_GUARD_WORKSPACES): a kernel that writes
+// outside a workspace is caught by ta_test_check_guards instead of corrupting its neighbour silently.
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardFill = 0xA5;
+thread_local std::vector<GuardRec> *g_guard_sink = nullptr;      // set while ta_create allocates for a guarded handle
+
 template <typename T> cudaError_t dev_alloc(T **p, size_t count)
 {
-    return cudaMalloc(reinterpret_cast<void **>(p), std::max<size_t>(count, 1) * sizeof(T));
+    const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
+    if (!g_guard_sink) return cudaMalloc(reinterpret_cast<void **>(p), bytes);
+    char *raw = nullptr;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&raw), bytes + 2 * kGuardBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaMemset(raw, kGuardFill, kGuardBytes);
+    if (e == cudaSuccess) e = cudaMemset(raw + kGuardBytes + bytes, kGuardFill, kGuardBytes);
+    *p = reinterpret_cast<T *>(raw + kGuardBytes);
+    g_guard_sink->push_back(GuardRec{raw, *p, bytes});
+    return e;
 }
 
-void free_all(DeviceBuffers &d)
+void free_all(DeviceBuffers &d, const std::vector<GuardRec> &guards = {})
 {
     void *ptrs[] = {d.pipe_tasks_sweep, d.pipe_tasks_apply, d.pipe_tasks_hold, d.pipe_batch_lo, d.pipe_bsum, d.pipe_layer_done, d.pipe_layer_ready, d.pipe_ctl,
                     d.warp_head, d.block_head, d.block_layer, d.slot_table, d.part, d.mom, d.pw_part, d.pw_coef, d.pw_norm, d.barrier, d.items, d.item_lo, d.seg_off, d.seg_len, d.seg_k, d.state, d.scratch, d.status, d.p_s1, d.p_s2, d.p_piv,
                     d.p_sa, d.p_mass, d.p_amax, d.p_amin, d.p_bad, d.window, d.hist, d.sel, d.mask, d.cand_count, d.cand_val, d.cand_idx, d.batch_seg, d.st_w, d.st_hz,
                     d.st_g, d.st_c};
-    for (void *p : ptrs)
-        if (p) cudaFree(p);
+    for (void *p : ptrs) {
+        if (!p) continue;
+        void *raw = p;
+        for (const GuardRec &g : guards)
+            if (g.user == p) raw = g.raw;
+        cudaFree(raw);
+    }
     d = DeviceBuffers{};
 }
 
@@ -454,7 +480,7 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
     if (hp->grad_dtype != TA_GRAD_F32 && hp->grad_dtype != TA_GRAD_BF16) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown grad_dtype");
     if (!(hp->momentum >= 0.f && hp->momentum < 1.f)) return fail(nullptr, TA_ERR_ARG, "ta_create: momentum must be in [0,1)");
     if (!(hp->weight_decay >= 0.f) || !(hp->weight_decay < 1e30f)) return fail(nullptr, TA_ERR_ARG, "ta_create: weight_decay must be finite and >= 0");
-    if (hp->flags & ~(uint32_t)(TA_FLAG_INPUTS_FINITE | TA_FLAG_NO_ONE_LAUNCH)) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown bit in flags");
+    if (hp->flags & ~(uint32_t)(TA_FLAG_INPUTS_FINITE | TA_FLAG_NO_ONE_LAUNCH | TA_FLAG_GUARD_WORKSPACES)) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown bit in flags");
     if (n_total % 4 != 0) return fail(nullptr, TA_ERR_ARG, "ta_create: n_total must be a multiple of 4");
     uint64_t end = 0, n_params = 0;
     for (uint32_t l = 0; l < L; ++l) {
@@ -475,10 +501,12 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
     if (!h) return fail(nullptr, TA_ERR_NOMEM, "ta_create: out of host memory");
     auto bail = [&](int code) {
         snprintf(g_create_error, 256, "%s", h->err);
-        free_all(h->d);
+        g_guard_sink = nullptr;
+        free_all(h->d, h->guards);
         delete h;
         return code;
     };
+    if (hp->flags & TA_FLAG_GUARD_WORKSPACES) g_guard_sink = &h->guards;
 #define TA_TRY(call)                                                                 \
     do {                                                                             \
         cudaError_t e__ = (call);                                                    \
@@ -718,6 +746,7 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
     }
     TA_TRY(cudaDeviceSynchronize());
 #undef TA_TRY
+    g_guard_sink = nullptr;
     *out = h;
     return TA_OK;
 }
@@ -744,7 +773,7 @@ int ta_destroy(ta_handle *h)
     if (h->copy_back) { cudaStreamSynchronize(h->copy_back); cudaStreamDestroy(h->copy_back); }
     for (cudaEvent_t e : h->chunk_done) cudaEventDestroy(e);
     if (h->decided) cudaEventDestroy(h->decided);
-    free_all(h->d);
+    free_all(h->d, h->guards);
     cudaSetDevice(prev);
     delete h;
     return TA_OK;
@@ -770,6 +799,26 @@ int ta_test_expire_next_wait(ta_handle *h)
     if (!h) return TA_ERR_ARG;
     if (!h->fused_ok) return fail(h, TA_ERR_STATE, "ta_test_expire_next_wait: this handle does not use the one-launch path");
     h->expire_next_wait = true;
+    return TA_OK;
+}
+
+int ta_test_check_guards(ta_handle *h)
+{
+    if (!h) return TA_ERR_ARG;
+    if (!(h->hp.flags & TA_FLAG_GUARD_WORKSPACES)) return fail(h, TA_ERR_STATE, "ta_test_check_guards: the handle was created without TA_FLAG_GUARD_WORKSPACES");
+    TA_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    unsigned char host[2 * kGuardBytes];
+    for (size_t i = 0; i < h->guards.size(); ++i) {
+        const GuardRec &g = h->guards[i];
+        TA_CUDA(h, cudaMemcpy(host, g.raw, kGuardBytes, cudaMemcpyDeviceToHost));
+        TA_CUDA(h, cudaMemcpy(host + kGuardBytes, static_cast<char *>(g.raw) + kGuardBytes + g.bytes, kGuardBytes, cudaMemcpyDeviceToHost));
+        for (size_t b = 0; b < 2 * kGuardBytes; ++b) {
+            if (host[b] != (unsigned char)kGuardFill) {
+                snprintf(h->err, 256, "a guard word %s workspace %zu (%zu bytes) was overwritten", b < kGuardBytes ? "in front of" : "behind", i, g.bytes);
+                return TA_ERR_STATE;
+            }
+        }
+    }
     return TA_OK;
 }
 

@@ -141,7 +141,8 @@ class ParityRun:
         self.table, self.n_total, self.hp = list(table), int(n_total), dict(hp)
         self.layers = list(range(len(table))) if layers is None else list(layers)
         self.sub_table = [self.table[l] for l in self.layers]
-        self.h = ta.ta_create(self.table, self.n_total, **self.hp)
+        # every workspace of the library between guard words, checked after each compared step
+        self.h = ta.ta_create(self.table, self.n_total, **dict(self.hp, flags=self.hp.get("flags", 0) | ta.TA_FLAG_GUARD_WORKSPACES))
         threads = min(int(threads), os.cpu_count() or 1)
         ohp = {k: v for k, v in self.hp.items() if k != "flags"}      # flags choose among CUDA paths; the method is the same
         self.o = (orc.Oracle(self.sub_table, self.n_total, **ohp) if threads <= 1 else
@@ -170,6 +171,7 @@ class ParityRun:
 
     def check(self, t):
         stats, status = ta.ta_stats(self.h)
+        ta.ta_test_check_guards(self.h)
         ost = self.o.status()
         full = len(self.layers) == len(self.table)
         if full:

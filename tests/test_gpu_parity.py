@@ -49,13 +49,13 @@ def test_mlp_tiny_unpadded_offsets():
 
 def test_resnet18_cifar_all_steps():
     wl = W.get("resnet18_cifar")
-    run = run_workload(wl, wl.steps, check_every=10)
+    run = run_workload(wl, wl.steps, check_every=10, threads=8)
     assert set(int(c) for c in run.o.codes()) == {0, 1, 2}    # FP16, BF16 and FP32 layers all occur
 
 
 def test_efficientnet_b0_all_steps():
     wl = W.get("efficientnet_b0_cifar")
-    run_workload(wl, wl.steps, check_every=10)
+    run_workload(wl, wl.steps, check_every=10, threads=8)
 
 
 def test_efficientnet_b0_unpadded_offsets():
@@ -65,7 +65,7 @@ def test_efficientnet_b0_unpadded_offsets():
 def test_resnet50_topk_full_size_all_steps():
     # all 50 steps at full size; the oracle runs one instance per host thread over a share of the layers
     wl = W.get("resnet50_topk")
-    run_workload(wl, wl.steps, check_every=5, threads=8)
+    run_workload(wl, wl.steps, check_every=5, threads=16)
 
 
 def test_resnet50_topk_quarter_width_curvature_every_third_step():
@@ -84,7 +84,7 @@ def test_gpt_1p3b_all_steps_sampled_layers():
     w0 = W.make_weights(wl, "cuda")
     D_dev = W.make_curvature(wl, "cuda")
     D_host = {l: D_dev[wl.table[l][0]:wl.table[l][0] + wl.table[l][1]].cpu().numpy() for l in layers}
-    run = ParityRun(wl.table, wl.n_total, wl.hparams(), w0, layers=layers, threads=8)
+    run = ParityRun(wl.table, wl.n_total, wl.hparams(), w0, layers=layers, threads=16)
     del w0
     z = torch.empty(wl.n_total, device="cuda")
     for t in range(1, wl.steps + 1):

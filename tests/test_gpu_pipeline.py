@@ -88,4 +88,4 @@ def test_flag_is_accepted_where_the_pipelined_pass_does_not_apply():
     assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32)) and torch.equal(outs[0][1], outs[1][1])
     assert outs[0][2] == outs[1][2] == 2
     with pytest.raises(ta.TriAccelError):
-        ta.ta_create(wl.table, wl.n_total, flags=4)
+        ta.ta_create(wl.table, wl.n_total, flags=8)
