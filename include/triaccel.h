@@ -113,6 +113,14 @@ typedef struct {
  * number in ta_last_error).  Results and speed of the pass are unchanged.
  */
 #define TA_FLAG_GUARD_WORKSPACES 4u
+/*
+ * TA_FLAG_COOPERATIVE_LAUNCH -- small dense models run the pass as two dependent launches over one plan (statistics;
+ * decisions and update), the second waiting for the first in hardware and the first launch of the next step free to
+ * start beside the second of this one.  With this flag they run as ONE cooperative launch around a grid-wide barrier
+ * instead, which keeps weights and gradients in shared memory between the two halves (models whose tensors fit).
+ * Same results.
+ */
+#define TA_FLAG_COOPERATIVE_LAUNCH 8u
 
 /* Per-layer statistics as of the last ta_step (host side, filled by ta_stats). */
 typedef struct {
@@ -286,6 +294,9 @@ int ta_shard_sweep(ta_handle *h, const void *g_local, const float *Hz_local, uin
 int ta_shard_apply(ta_handle *h, float *w_local, const void *g_local, uint16_t *c_local,
                    const ta_layer_record *records_all /* device, world * L records, rank-major */, uint32_t world, void *stream);
 
+/* How this handle runs the pass, in words (static string): "separate kernels", "two dependent launches", ... */
+const char *ta_path(const ta_handle *h);
+
 /* Number of kernels the library launched on behalf of this handle so far (for benchmarks). */
 int ta_launch_count(ta_handle *h, uint64_t *count);
 
@@ -299,8 +310,8 @@ int ta_timing_begin(ta_handle *h, uint32_t max_steps);
 int ta_timing_end(ta_handle *h, double *ms_sweep, double *ms_decide, double *ms_update, uint32_t *steps);
 
 /*
- * Failure detection.  Small dense models run as one cooperative launch whose blocks meet at a
- * grid-wide barrier.  Every such wait is bounded (a few hundred milliseconds): a block that gives up
+ * Failure detection.  With TA_FLAG_COOPERATIVE_LAUNCH small dense models run as one cooperative launch whose blocks
+ * meet at a grid-wide barrier.  Every such wait is bounded (a few hundred milliseconds): a block that gives up
  * records it and returns, the step then changes neither weights, copies nor per-layer state, and the
  * next ta_stats / ta_precision_codes returns TA_ERR_CUDA once ("a bounded device-side wait ran out"),
  * after which the handle is usable again.  ta_test_expire_next_wait is a test aid: it makes the waits of

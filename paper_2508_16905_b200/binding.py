@@ -16,14 +16,14 @@ LIB_PATH = os.path.join(HERE, "libtriaccel.so")
 TA_OK, TA_ERR_ARG, TA_ERR_ALIGN, TA_ERR_STATE, TA_ERR_CUDA, TA_ERR_NOMEM = 0, -1, -2, -3, -4, -5
 TA_CODE_FP16, TA_CODE_BF16, TA_CODE_FP32 = 0, 1, 2
 TA_GRAD_F32, TA_GRAD_BF16 = 0, 1
-TA_FLAG_INPUTS_FINITE, TA_FLAG_NO_ONE_LAUNCH, TA_FLAG_GUARD_WORKSPACES = 1, 2, 4
+TA_FLAG_INPUTS_FINITE, TA_FLAG_NO_ONE_LAUNCH, TA_FLAG_GUARD_WORKSPACES, TA_FLAG_COOPERATIVE_LAUNCH = 1, 2, 4, 8
 
 EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "ta_probe", "ta_stats",
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
            "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
            "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait",
            "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch", "ta_plan_pipeline",
-           "ta_create_shard", "ta_shard_sweep", "ta_shard_apply", "ta_test_check_guards"]
+           "ta_create_shard", "ta_shard_sweep", "ta_shard_apply", "ta_test_check_guards", "ta_path"]
 
 
 class ta_segment(C.Structure):
@@ -107,6 +107,8 @@ def lib():
     L.ta_grad_moments_static.argtypes = [C.POINTER(ta_segment), u32, vp, u32, vp, vp, vp]
     L.ta_test_expire_next_wait.argtypes = [vp]
     L.ta_test_check_guards.argtypes = [vp]
+    L.ta_path.argtypes = [vp]
+    L.ta_path.restype = C.c_char_p
     L.ta_power_iterate.argtypes = [vp, vp, vp, vp, vp, u32, vp, vp, vp, vp]
     L.ta_set_curvature.argtypes = [vp, vp]
     L.ta_plan_one_launch.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_run), u32, C.POINTER(u32), C.POINTER(u32),
@@ -118,7 +120,7 @@ def lib():
     L.ta_static_last_error.argtypes = []
     L.ta_static_last_error.restype = C.c_char_p
     for name in EXPORTS:
-        if name not in ("ta_last_error", "ta_static_last_error"):
+        if name not in ("ta_last_error", "ta_static_last_error", "ta_path"):
             getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -130,11 +132,17 @@ def _check(rc, h=None):
 
 
 def _dev_ptr(t):
-    if t is None:
-        return None
+    if t is None or isinstance(t, C.c_void_p):      # already marshalled (callers in a hurry wrap their tensors once: dev_ptr)
+        return t
     if not t.is_cuda or not t.is_contiguous():
         raise ValueError("device buffers must be contiguous CUDA tensors")
     return C.c_void_p(t.data_ptr())
+
+
+def dev_ptr(t):
+    """The device address of a contiguous CUDA tensor, marshalled once, for callers that pass the same buffers to many
+    calls (every ta_* function takes it in place of the tensor; the tensor must stay alive)."""
+    return _dev_ptr(t)
 
 
 def _host_ptr(a):
@@ -151,6 +159,8 @@ def _stream(stream):
     if stream is None:
         import torch
         return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, C.c_void_p):
+        return stream
     return C.c_void_p(int(stream))
 
 
@@ -345,6 +355,10 @@ def ta_plan_pipeline(table, with_decisions=True):
     if rc != TA_OK:
         raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
     return [(t.kind, t.layer, t.begin, t.length) for t in out[:n.value]]
+
+
+def ta_path(h):
+    return (lib().ta_path(h.ptr) or b"").decode()
 
 
 def ta_test_check_guards(h):

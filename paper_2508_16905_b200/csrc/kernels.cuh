@@ -1265,7 +1265,8 @@ struct FusedArgs {
     uint32_t max_block_layers;          // layers of the block that touches most layers
     uint32_t early_weights;             // 1: the weight copies start with the first loads of the sweep, 0: after the sweep
     unsigned long long step;
-    unsigned long long *barrier;        // [0] arrivals, only ever incremented; [1] last launch that saw non-finite input
+    unsigned long long *barrier;        // [0] arrivals, only ever incremented
+    unsigned long long *flag;           // number of the last launch that saw non-finite input
     unsigned long long barrier_base;    // arrivals before this launch
     unsigned long long epoch;           // number of this launch (from 1)
 };
@@ -1335,10 +1336,24 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsign
     return ok != 0u;
 }
 
-template <int P, bool BF16>
+// Dependencies between consecutive launches of one stream that the hardware resolves (no spinning): a launch may
+// start while its predecessor still runs, and waits here until the predecessor is complete and its writes are visible.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// From here on the next launch of the stream may start.
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// MODE 0: the whole step in one cooperative launch.  The same step as two dependent launches over the same plan, with
+// nothing kept in shared memory between them: MODE 1 is the sweep (statistics and block partials), MODE 2 the decisions
+// and the update.  The sweep of step t + 1 needs nothing from the update of step t, so it may run beside it; it only
+// ends after it (so that "the update of step t + 1 has waited for its sweep" also means "... and for the update of
+// step t").  Partials and the non-finite flag alternate between two buffers for that reason.
+constexpr int kWholeStep = 0, kSweepHalf = 1, kUpdateHalf = 2;
+
+template <int P, bool BF16, int MODE>
 __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <= 4 ? 2 : 1))) k_fused(const FusedArgs A)
 {
     constexpr int PP = P > 0 ? P : 1;
+    if (MODE == kSweepHalf) grid_dependency_release();      // the update half may take its places and read its plan
     constexpr int U = (P <= 1) ? TA_FUSED_SWEEP_SLOTS : (P == 2 ? 4 : 2);     // slots in flight per lane during the sweep
     constexpr int UA = TA_FUSED_UPDATE_SLOTS;                                  // slots per group of the update
     extern __shared__ __align__(16) unsigned char dyn_smem[];
@@ -1383,8 +1398,15 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
     // anybody can have written a new one
     for (uint32_t i = tid; i < nl * 2u; i += kThreads)
         cp_async16(reinterpret_cast<uint4 *>(sh_bl) + i, reinterpret_cast<const uint4 *>(A.block_layer + bpart_lo) + i);
-    for (uint32_t i = tid; i < nl * kStateWords; i += kThreads)
-        cp_async8(sh_old + i, reinterpret_cast<const unsigned long long *>(A.state + lf) + i);
+    if (MODE == kUpdateHalf) {
+        // everything above is the plan, which no launch writes; what follows needs the sweep of this step (and, through
+        // it, the update of the step before) complete.  Then the sweep of the next step may start.
+        grid_dependency_wait();
+        grid_dependency_release();
+    }
+    if (MODE != kSweepHalf)
+        for (uint32_t i = tid; i < nl * kStateWords; i += kThreads)
+            cp_async8(sh_old + i, reinterpret_cast<const unsigned long long *>(A.state + lf) + i);
     cp_async_commit();
     __syncwarp();
 
@@ -1396,7 +1418,7 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
     };
 
     // phase 1: statistics of this warp's runs (Sec. 3.1 moments; Sec. 3.2 probe sums)
-    {
+    if constexpr (MODE != kUpdateHalf) {
         SweepAcc<P, false> acc;
         uint32_t X[PP][4];
         uint64_t have_block = ~0ull;
@@ -1502,9 +1524,12 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
             }
         }
         if (n_slots) flush(cur_run);
-        // the weights arrive while the grid waits at the barrier and takes the decisions
-        if (!A.early_weights || n_slots == 0) start_weight_copies();
-        if (bad_seen && lane == 0) atomicMax(A.barrier + 1, A.epoch);
+        if (MODE == kSweepHalf) {
+            // nothing to start: the update half reads the weights itself
+        } else if (!A.early_weights || n_slots == 0) {
+            start_weight_copies();      // the weights arrive while the grid waits at the barrier and takes the decisions
+        }
+        if (bad_seen && lane == 0) atomicMax(A.flag, A.epoch);
     }
     // decisions of one layer of this block, from the layer's sums over all blocks (Sec. 3.1 - 3.4).  The new state
     // replaces the old one in shared memory; the block that holds the layer's first run writes it out once the step
@@ -1654,30 +1679,38 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
     };
 
     // the block's runs folded into one partial per layer it touches, in run order
-    cp_async_wait_but_one();        // the block's tables have arrived (the weight copies may still be under way)
+    if (MODE == kUpdateHalf) cp_async_wait_all();
+    else cp_async_wait_but_one();   // the block's tables have arrived (the weight copies may still be under way)
     __syncthreads();
-    for (uint32_t q = tid; q < nl; q += kThreads) {
-        const uint32_t lo = sh_bl[q].run_lo, hi = sh_bl[q].run_hi;
-        FusedPartial t{0.0, 0.0, 0u, 0xFFFFFFFFu, 0u, sh_run[lo - brun_lo].pivot, 0u, 0u};
-        for (uint32_t r = lo; r < hi; ++r) {
-            const FusedPartial x = sh_run[r - brun_lo];
-            const MomentSums m = rebase(x.s1, x.s2, (double)x.n, (double)x.pivot, (double)t.pivot);
-            t.s1 += m.s1; t.s2 += m.s2;
-            t.n += x.n;
-            t.amax = max(t.amax, x.amax); t.amin = min(t.amin, x.amin);
-            t.bad += x.bad;
+    if constexpr (MODE != kUpdateHalf) {
+        for (uint32_t q = tid; q < nl; q += kThreads) {
+            const uint32_t lo = sh_bl[q].run_lo, hi = sh_bl[q].run_hi;
+            FusedPartial t{0.0, 0.0, 0u, 0xFFFFFFFFu, 0u, sh_run[lo - brun_lo].pivot, 0u, 0u};
+            for (uint32_t r = lo; r < hi; ++r) {
+                const FusedPartial x = sh_run[r - brun_lo];
+                const MomentSums m = rebase(x.s1, x.s2, (double)x.n, (double)x.pivot, (double)t.pivot);
+                t.s1 += m.s1; t.s2 += m.s2;
+                t.n += x.n;
+                t.amax = max(t.amax, x.amax); t.amin = min(t.amin, x.amin);
+                t.bad += x.bad;
+            }
+            A.part[bpart_lo + q] = t;
         }
-        A.part[bpart_lo + q] = t;
+    }
+    if (MODE == kSweepHalf) {
+        // this launch is complete only when the update of the step before is (see kSweepHalf above)
+        grid_dependency_wait();
+        return;
     }
 
-    if (!grid_barrier(A.barrier, A.barrier_base + G, A.status)) {
+    if (MODE == kWholeStep && !grid_barrier(A.barrier, A.barrier_base + G, A.status)) {
         cp_async_wait_all();
         return;
     }
 
     // did any warp of the grid see a non-finite input?  The answer is needed only when results are committed, so
     // the decisions below are taken while it is on its way; those of a skipped step are thrown away
-    const bool skip = __ldcg(A.barrier + 1) == A.epoch || __ldcg(&A.status->device_error) != 0u;
+    const bool skip = __ldcg(A.flag) == A.epoch || __ldcg(&A.status->device_error) != 0u;
     for (uint32_t q = tid; q < nl; q += kThreads) {
         const uint32_t lo = sh_bl[q].part_lo, hi = sh_bl[q].part_hi;
         if (hi - lo <= kThreadCombine) combine_serial(q, lo, hi);

@@ -79,7 +79,8 @@ struct ta_handle {
     std::vector<cudaEvent_t> events;      // 4 per timed step: before sweep, after sweep, after decisions, after update
     uint32_t timed_cap = 0, timed_used = 0;
     bool expire_next_wait = false;        // test aid: the next one-launch step waits for arrivals that never come
-    bool fused_ok = false;                // small dense models: sweep + decisions + update in one cooperative launch
+    bool fused_ok = false;                // small dense models: sweep + decisions + update in one cooperative launch ...
+    bool fused_split = false;             // ... or as two dependent launches over the same plan (the default)
     int fused_grid = 0;                   // blocks of the one-launch grid (all resident)
     uint32_t fused_cap_w = 0, fused_cap_g = 0;                           // shared-memory slots per warp: weights, gradients
     uint32_t fused_block_layers = 0, fused_block_runs = 0, fused_slots = 0, fused_parts = 0;   // table sizes of the plan
@@ -230,19 +231,22 @@ void launch_apply(ta_handle *h, float *w, const void *g, uint16_t *c, uint32_t i
     ++h->launches;
 }
 
-template <int P, bool BF16> const void *fused_fn() { return reinterpret_cast<const void *>(&ta::k_fused<P, BF16>); }
+template <int P, bool BF16, int MODE> const void *fused_fn() { return reinterpret_cast<const void *>(&ta::k_fused<P, BF16, MODE>); }
 
-const void *fused_kernel(int P, bool bf16)
+template <int MODE> const void *fused_kernel_mode(int P, bool bf16)
 {
     switch (P) {
-    case 0: return bf16 ? fused_fn<0, true>() : fused_fn<0, false>();
-    case 1: return bf16 ? fused_fn<1, true>() : fused_fn<1, false>();
-    case 2: return bf16 ? fused_fn<2, true>() : fused_fn<2, false>();
-    case 4: return bf16 ? fused_fn<4, true>() : fused_fn<4, false>();
-    case 8: return bf16 ? fused_fn<8, true>() : fused_fn<8, false>();
+    case 0: return bf16 ? fused_fn<0, true, MODE>() : fused_fn<0, false, MODE>();
+    case 1: return bf16 ? fused_fn<1, true, MODE>() : fused_fn<1, false, MODE>();
+    case 2: return bf16 ? fused_fn<2, true, MODE>() : fused_fn<2, false, MODE>();
+    case 4: return bf16 ? fused_fn<4, true, MODE>() : fused_fn<4, false, MODE>();
+    case 8: return bf16 ? fused_fn<8, true, MODE>() : fused_fn<8, false, MODE>();
     default: return nullptr;
     }
 }
+const void *fused_kernel(int P, bool bf16) { return fused_kernel_mode<ta::kWholeStep>(P, bf16); }
+const void *sweep_half_kernel(int P, bool bf16) { return fused_kernel_mode<ta::kSweepHalf>(P, bf16); }
+const void *update_half_kernel(bool bf16) { return bf16 ? fused_fn<0, true, ta::kUpdateHalf>() : fused_fn<0, false, ta::kUpdateHalf>(); }
 
 constexpr int kFusedSmemMax = 226 * 1024;         // dynamic shared memory a block may ask for (227 KB opt-in limit minus the static part)
 constexpr uint64_t kRunOverhead = 256;            // cost of starting a run, in elements: reductions and partial rows
@@ -426,7 +430,7 @@ int check_device_error(ta_handle *h)
     if (!s.device_error) return TA_OK;
     s.device_error = 0u;
     TA_CUDA(h, cudaMemcpy(h->d.status, &s, sizeof(s), cudaMemcpyHostToDevice));
-    if (h->d.barrier) TA_CUDA(h, cudaMemset(h->d.barrier, 0, 2 * sizeof(unsigned long long)));
+    if (h->d.barrier) TA_CUDA(h, cudaMemset(h->d.barrier, 0, 4 * sizeof(unsigned long long)));
 
     h->barrier_base = 0;
     h->fused_launches = 0;
@@ -480,7 +484,7 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
     if (hp->grad_dtype != TA_GRAD_F32 && hp->grad_dtype != TA_GRAD_BF16) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown grad_dtype");
     if (!(hp->momentum >= 0.f && hp->momentum < 1.f)) return fail(nullptr, TA_ERR_ARG, "ta_create: momentum must be in [0,1)");
     if (!(hp->weight_decay >= 0.f) || !(hp->weight_decay < 1e30f)) return fail(nullptr, TA_ERR_ARG, "ta_create: weight_decay must be finite and >= 0");
-    if (hp->flags & ~(uint32_t)(TA_FLAG_INPUTS_FINITE | TA_FLAG_NO_ONE_LAUNCH | TA_FLAG_GUARD_WORKSPACES)) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown bit in flags");
+    if (hp->flags & ~(uint32_t)(TA_FLAG_INPUTS_FINITE | TA_FLAG_NO_ONE_LAUNCH | TA_FLAG_GUARD_WORKSPACES | TA_FLAG_COOPERATIVE_LAUNCH)) return fail(nullptr, TA_ERR_ARG, "ta_create: unknown bit in flags");
     if (n_total % 4 != 0) return fail(nullptr, TA_ERR_ARG, "ta_create: n_total must be a multiple of 4");
     uint64_t end = 0, n_params = 0;
     for (uint32_t l = 0; l < L; ++l) {
@@ -543,11 +547,19 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
             n_params <= kFusedMaxParams) {
             const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
             h->fused_ok = true;
+            h->fused_split = !(hp->flags & TA_FLAG_COOPERATIVE_LAUNCH);
             fused_per_sm = 1 << 20;
             for (int P : {0, (int)hp->num_probes}) {
                 int per_sm = 0;
-                TA_TRY(cudaFuncSetAttribute(fused_kernel(P, bf16), cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemMax));
-                TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(P, bf16), ta::kThreads, 0));
+                const void *fn = h->fused_split ? sweep_half_kernel(P, bf16) : fused_kernel(P, bf16);
+                TA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemMax));
+                TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, ta::kThreads, 0));
+                fused_per_sm = std::min(fused_per_sm, per_sm);
+            }
+            if (h->fused_split) {
+                int per_sm = 0;
+                TA_TRY(cudaFuncSetAttribute(update_half_kernel(bf16), cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemMax));
+                TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, update_half_kernel(bf16), ta::kThreads, 0));
                 fused_per_sm = std::min(fused_per_sm, per_sm);
             }
             if (fused_per_sm < 1) h->fused_ok = false;
@@ -583,6 +595,7 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
             h->fused_cap_w = (uint32_t)std::min<long long>(pl.max_slots, rows_fit);
             h->fused_cap_g = (uint32_t)std::min<long long>(pl.max_slots, rows_fit - h->fused_cap_w);
             if (h->fused_cap_w < pl.max_slots) h->fused_cap_w = h->fused_cap_g = 0;
+            if (h->fused_split) h->fused_cap_w = h->fused_cap_g = 0;      // nothing survives in shared memory between two launches
             h->fused_block_layers = pl.max_block_layers;
             h->fused_block_runs = pl.max_block_runs;
             h->fused_slots = pl.max_slots;
@@ -687,8 +700,8 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
         TA_TRY(cudaMemset(d.mom, 0, n_total * sizeof(float)));
     }
     if (h->fused_ok) {
-        TA_TRY(dev_alloc(&d.barrier, 2));
-        TA_TRY(cudaMemset(d.barrier, 0, 2 * sizeof(unsigned long long)));
+        TA_TRY(dev_alloc(&d.barrier, 4));          // arrivals, non-finite flag; two more flags for the two-launch form
+        TA_TRY(cudaMemset(d.barrier, 0, 4 * sizeof(unsigned long long)));
 
         TA_TRY(dev_alloc(&d.warp_head, run_plan.warp_head.size()));
         TA_TRY(cudaMemcpy(d.warp_head, run_plan.warp_head.data(), run_plan.warp_head.size() * sizeof(ta::FusedWarpHead), cudaMemcpyHostToDevice));
@@ -698,12 +711,12 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
         TA_TRY(cudaMemcpy(d.block_layer, run_plan.block_layer.data(), run_plan.block_layer.size() * sizeof(ta::FusedBlockLayer), cudaMemcpyHostToDevice));
         TA_TRY(dev_alloc(&d.slot_table, run_plan.slot_table.size()));
         TA_TRY(cudaMemcpy(d.slot_table, run_plan.slot_table.data(), run_plan.slot_table.size() * sizeof(ta::FusedSlot), cudaMemcpyHostToDevice));
-        TA_TRY(dev_alloc(&d.part, h->fused_parts));
+        TA_TRY(dev_alloc(&d.part, 2 * (size_t)h->fused_parts));      // the two-launch form alternates between two sets
         // the occupancy the plan counted on must hold with the shared memory it asks for
         const bool bf16 = hp->grad_dtype == TA_GRAD_BF16;
         for (int P : {0, (int)hp->num_probes}) {
             int per_sm = 0;
-            TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(P, bf16), ta::kThreads, h->fused_smem));
+            TA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, h->fused_split ? sweep_half_kernel(P, bf16) : fused_kernel(P, bf16), ta::kThreads, h->fused_smem));
             if ((long long)per_sm * h->sm_count < h->fused_grid) {
                 snprintf(h->err, 256, "ta_create: the one-launch grid of %d blocks is not resident (%d per SM)", h->fused_grid, per_sm);
                 return bail(TA_ERR_CUDA);
@@ -787,6 +800,15 @@ int ta_set_lr(ta_handle *h, float eta0)
     return TA_OK;
 }
 
+const char *ta_path(const ta_handle *h)
+{
+    if (!h) return "";
+    if (h->sharded) return "sharded: sweep, record exchange, update";
+    if (h->pipe_ok) return "pipelined launch";
+    if (h->fused_ok) return h->fused_split ? "two dependent launches" : "one cooperative launch";
+    return h->topk ? "separate kernels with top-k selection" : "separate kernels";
+}
+
 int ta_launch_count(ta_handle *h, uint64_t *count)
 {
     if (!h || !count) return TA_ERR_ARG;
@@ -797,7 +819,7 @@ int ta_launch_count(ta_handle *h, uint64_t *count)
 int ta_test_expire_next_wait(ta_handle *h)
 {
     if (!h) return TA_ERR_ARG;
-    if (!h->fused_ok) return fail(h, TA_ERR_STATE, "ta_test_expire_next_wait: this handle does not use the one-launch path");
+    if (!h->fused_ok || h->fused_split) return fail(h, TA_ERR_STATE, "ta_test_expire_next_wait: this handle does not use the one-launch path");
     h->expire_next_wait = true;
     return TA_OK;
 }
@@ -963,8 +985,33 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
         fa.dp.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; fa.dp.topk = 0u;
         fa.L = h->L; fa.cap_w = h->fused_cap_w; fa.cap_g = h->fused_cap_g;
         fa.max_slots = h->fused_slots; fa.max_block_runs = h->fused_block_runs; fa.max_block_layers = h->fused_block_layers;
-        fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base;
+        fa.step = step; fa.barrier = d.barrier; fa.barrier_base = h->barrier_base; fa.flag = d.barrier + 1;
         fa.epoch = h->fused_launches + 1;
+        if (h->fused_split) {
+            // two dependent launches: the sweep of this step may run beside the update of the step before (it touches
+            // none of its data), so partials and the non-finite flag alternate between two sets
+            const unsigned long long parity = h->fused_launches & 1ull;
+            fa.part = d.part + parity * h->fused_parts;
+            fa.flag = d.barrier + 2 + parity;
+            fa.early_weights = 0u;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)h->fused_grid); cfg.blockDim = dim3(ta::kThreads);
+            cfg.dynamicSmemBytes = h->fused_smem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
+            void *args[] = {&fa};
+            TA_CUDA(h, cudaLaunchKernelExC(&cfg, sweep_half_kernel(P, bf16), args));
+            if (timed) { cudaEventRecord(ev[1], s); cudaEventRecord(ev[2], s); }
+            TA_CUDA(h, cudaLaunchKernelExC(&cfg, update_half_kernel(bf16), args));
+            ++h->fused_launches;
+            h->launches += 2;
+            if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
+            h->stepped = true;
+            h->last_step = step;
+            h->last_stream = s;
+            return TA_OK;
+        }
         fa.early_weights = 0u;
       // the weight copies start after the sweep (measured faster than starting them with its first loads)
         if (h->expire_next_wait) { fa.barrier_base += 1ull << 40; h->expire_next_wait = false; }

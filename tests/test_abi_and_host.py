@@ -52,7 +52,7 @@ def test_create_rejects_bad_arguments_before_touching_a_device():
         dict(table=[(0, 8)], n_total=8, t_ctrl=0),
         dict(table=[(0, 8)], n_total=8, momentum=1.0),
         dict(table=[(0, 8)], n_total=8, weight_decay=-1.0),
-        dict(table=[(0, 8)], n_total=8, flags=8),                # unknown flag bit
+        dict(table=[(0, 8)], n_total=8, flags=16),               # unknown flag bit
         dict(table=[(0, 8)], n_total=8, tau_low=2.0, tau_high=1.0),
     ]
     for kw in bad:

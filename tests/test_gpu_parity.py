@@ -58,6 +58,17 @@ def test_efficientnet_b0_all_steps():
     run_workload(wl, wl.steps, check_every=10, threads=8)
 
 
+@pytest.mark.parametrize("name", ["mlp_tiny", "efficientnet_b0_cifar", "resnet18_cifar"])
+def test_small_models_as_one_cooperative_launch(name):
+    wl = W.get(name)
+    w0 = W.make_weights(wl, "cuda")
+    D = W.make_curvature(wl, "cuda").cpu().numpy()
+    run = ParityRun(wl.table, wl.n_total, dict(wl.hparams(), flags=ta.TA_FLAG_COOPERATIVE_LAUNCH), w0, threads=8)
+    for t in range(1, 6):
+        run.step(t, W.make_grads(wl, t, "cuda"), oracle_hz(D, 1, wl.probe_seed, t) if t != 3 else None, wl.probe_seed)
+    assert ta.ta_path(run.h) == "one cooperative launch" and ta.ta_launch_count(run.h) == 5
+
+
 def test_efficientnet_b0_unpadded_offsets():
     run_workload(W.get("efficientnet_b0_cifar", align=1), 3)
 
@@ -211,7 +222,7 @@ def test_constant_gradient_has_zero_variance():
     assert s.grad_var == 0.0          # differences from the pivot are all zero
 
 
-@pytest.mark.parametrize("path", ["one_launch", "sweep"])
+@pytest.mark.parametrize("path", ["two dependent launches", "one cooperative launch", "separate kernels"])
 @pytest.mark.parametrize("grad_dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("ratio", [1e3, 1e5])
 def test_moments_of_gradients_with_a_large_mean(path, grad_dtype, ratio):
@@ -220,8 +231,8 @@ def test_moments_of_gradients_with_a_large_mean(path, grad_dtype, ratio):
     table, n_total = ragged_table([1500000, 70000, 1000, 33])
     rng = np.random.default_rng(int(ratio) + len(path))
     hp = dict(beta=0.5, eta0=1e-3, grad_dtype=grad_dtype, tau_low=1e-12, tau_high=1e-7)
-    if path == "sweep":
-        hp["momentum"] = 0.5          # the update with a momentum buffer runs as separate sweep / decide / update kernels
+    hp["flags"] = {"two dependent launches": 0, "one cooperative launch": ta.TA_FLAG_COOPERATIVE_LAUNCH,
+                   "separate kernels": ta.TA_FLAG_NO_ONE_LAUNCH}[path]
     run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
     D = rng.uniform(0.1, 1.0, n_total).astype(np.float32)
     means = np.repeat([1.0, -0.37, 3e-3, 250.0], [n for _, n in table])
@@ -233,7 +244,8 @@ def test_moments_of_gradients_with_a_large_mean(path, grad_dtype, ratio):
         if grad_dtype == "bf16":
             g_dev = g_dev.to(torch.bfloat16)
         run.step(t, g_dev, oracle_hz(D, 1, 5, t) if t != 2 else None, 5)
-    assert ta.ta_launch_count(run.h) == (3 if path == "one_launch" else 9)
+    assert ta.ta_path(run.h) == path
+    assert ta.ta_launch_count(run.h) == {"two dependent launches": 6, "one cooperative launch": 3, "separate kernels": 9}[path]
 
 
 def test_non_finite_input_skips_the_whole_step():
@@ -265,12 +277,14 @@ def test_non_finite_input_skips_the_whole_step():
     assert ta.ta_stats(run.h)[1].skipped == 0
 
 
-def test_non_finite_input_skips_the_whole_step_one_launch():
-    """Dense model on the one-launch path: bad values in a one-element layer, on the partial last row of a layer
-    and in two layers at once; the exact count is reported, nothing changes, and the next clean step matches."""
+@pytest.mark.parametrize("flags,per_step", [(0, 2), (ta.TA_FLAG_COOPERATIVE_LAUNCH, 1)])
+def test_non_finite_input_skips_the_whole_step_small_model(flags, per_step):
+    """Small dense model, as two dependent launches and as one cooperative launch: bad values in a one-element layer, on
+    the partial last row of a layer and in two layers at once; the exact count is reported, nothing changes, and the
+    next clean step matches."""
     table, n_total = ragged_table([1, 33, 5000, 2, 300, 70000, 129, 7])
     rng = np.random.default_rng(3)
-    hp = dict(num_probes=1, tau_low=3e-7, tau_high=3e-6)
+    hp = dict(num_probes=1, tau_low=3e-7, tau_high=3e-6, flags=flags)
     run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
     D = rng.uniform(0.1, 1.0, n_total).astype(np.float32)
 
@@ -299,7 +313,7 @@ def test_non_finite_input_skips_the_whole_step_one_launch():
         assert all(a.ema_var == b.ema_var and a.code == b.code and a.lambda_max == b.lambda_max for a, b in zip(stats, before[2]))
         t += 1
         assert run.step(t, grad(t), oracle_hz(D, 1, 0, t) if t % 4 else None, 0) is False       # and the pass goes on
-    assert ta.ta_launch_count(run.h) == t          # one launch per step
+    assert ta.ta_launch_count(run.h) == per_step * t
 
 
 def test_runs_are_bit_reproducible():
@@ -443,7 +457,7 @@ def test_bounded_wait_runs_out_without_hanging():
     g1, g2 = W.make_grads(wl, 1, "cuda"), W.make_grads(wl, 2, "cuda")
     hs, ws, cs = [], [], []
     for _ in range(2):
-        hs.append(ta.ta_create(wl.table, wl.n_total, **wl.hparams()))
+        hs.append(ta.ta_create(wl.table, wl.n_total, **wl.hparams(), flags=ta.TA_FLAG_COOPERATIVE_LAUNCH))
         ws.append(W.make_weights(wl, "cuda"))
         cs.append(torch.zeros(wl.n_total, dtype=torch.int16, device="cuda"))
         ta.ta_step(hs[-1], ws[-1], g1, None, cs[-1], 0, 1)

@@ -86,6 +86,6 @@ def test_flag_is_accepted_where_the_pipelined_pass_does_not_apply():
             ta.ta_step(h, w, W.make_grads(wl, t, "cuda"), None, c, 0, t)
         outs.append((w, c, ta.ta_launch_count(h)))
     assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32)) and torch.equal(outs[0][1], outs[1][1])
-    assert outs[0][2] == outs[1][2] == 2
+    assert outs[0][2] == outs[1][2] == 4           # two dependent launches per step either way
     with pytest.raises(ta.TriAccelError):
-        ta.ta_create(wl.table, wl.n_total, flags=8)
+        ta.ta_create(wl.table, wl.n_total, flags=16)
