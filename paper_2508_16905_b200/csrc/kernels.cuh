@@ -154,6 +154,13 @@ __device__ __forceinline__ uint32_t pick_word(const uint32_t (&x)[4], uint32_t j
 
 // ------------------------------------------------------------------ small helpers
 
+// Dependencies between consecutive launches of one stream that the hardware resolves (no spinning): a launch may
+// start while its predecessor still runs, and waits here until the predecessor is complete and its writes are visible.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// From here on the next launch of the stream may start.
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+
 __device__ __forceinline__ float4 ld_stream(const float *p)
 {
     return __ldcs(reinterpret_cast<const float4 *>(p));
@@ -770,6 +777,8 @@ __global__ void __launch_bounds__(kThreads, ((P == 4 || TOPK) && P <= 4 ? 2 : 1)
     __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
     __shared__ uint32_t sh_stage[TOPK ? kWarps * 2 * kStageCap : 1];
     extern __shared__ __align__(16) float4 sh_ring[];          // TOPK: kWarps * kSweepRing<P> rows of (1 + P) x 512 bytes
+    grid_dependency_wait();         // launched ahead of time: the kernel before this one is complete from here on
+    grid_dependency_release();
     if (TOPK && A.redo && (A.status->skipped || A.status->redo_layers == 0u)) return;      // nothing to repeat
     auto store = [&A](uint32_t it, const ItemSums &r) {
         A.p_s1[it] = r.s1;
@@ -945,6 +954,8 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     __shared__ uint32_t scan[kThreads];
     __shared__ uint32_t found[2];
     const uint32_t l = blockIdx.x, tid = threadIdx.x;
+    grid_dependency_wait();
+    grid_dependency_release();
     const uint32_t lo = A.item_lo[l], hi = A.item_lo[l + 1];
     if (A.topk) {
         // level-1 digit (bits 30..20) of the layer's k-th largest |S|; the histogram is cleared for the next
@@ -1176,6 +1187,8 @@ __device__ __forceinline__ void apply_batch(const ApplyArgs &A, uint32_t batch, 
 template <bool BF16, bool MOM>
 __global__ void __launch_bounds__(kThreads) k_apply(const ApplyArgs A)
 {
+    grid_dependency_wait();
+    grid_dependency_release();
     if (A.status->skipped) return;
     const LayerState *state = A.state;
     auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
@@ -1335,12 +1348,6 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long *counter, unsign
     __syncthreads();
     return ok != 0u;
 }
-
-// Dependencies between consecutive launches of one stream that the hardware resolves (no spinning): a launch may
-// start while its predecessor still runs, and waits here until the predecessor is complete and its writes are visible.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// From here on the next launch of the stream may start.
-__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // MODE 0: the whole step in one cooperative launch.  The same step as two dependent launches over the same plan, with
 // nothing kept in shared memory between them: MODE 1 is the sweep (statistics and block partials), MODE 2 the decisions
@@ -2061,6 +2068,8 @@ __device__ __forceinline__ void resolve_layer(const ResolveArgs &A, const uint32
 template <bool BF16, bool MOM>
 __global__ void __launch_bounds__(kThreads) k_apply_resolve(const ApplyArgs A, const ResolveArgs R, const uint32_t n_layers)
 {
+    grid_dependency_wait();
+    grid_dependency_release();
     if (A.status->skipped) return;
     if (blockIdx.x < n_layers) {
         resolve_layer(R, blockIdx.x);

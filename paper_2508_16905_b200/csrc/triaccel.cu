@@ -187,6 +187,21 @@ ta::Hyper hyper_of(const ta_hparams &hp)
     return y;
 }
 
+// Launches a kernel of the multi-kernel pass so that its blocks may be scheduled while the kernel before it in the
+// stream drains (its first instruction waits for that kernel's completion, so nothing else changes): the launch
+// latency between the three or four dependent kernels of a step is hidden behind the previous kernel's tail.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(void (*kernel)(KArgs...), unsigned grid, size_t smem, cudaStream_t s, Args... args)
+{
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(ta::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <int P, bool BF16, bool TOPK> void launch_sweep(ta_handle *h, const ta::SweepArgs &a, cudaStream_t s)
 {
     // the top-k sweeps stage their rows in a ring of shared memory (beyond the 48 KB a launch gets without asking)
@@ -198,7 +213,7 @@ template <int P, bool BF16, bool TOPK> void launch_sweep(ta_handle *h, const ta:
             asked = true;
         }
     }
-    ta::k_sweep<P, BF16, TOPK><<<grid_for(h), ta::kThreads, ring, s>>>(a);
+    launch_after(ta::k_sweep<P, BF16, TOPK>, (unsigned)grid_for(h), ring, s, a);
     ++h->launches;
 }
 
@@ -224,10 +239,10 @@ void launch_apply(ta_handle *h, float *w, const void *g, uint16_t *c, uint32_t i
                      h->d.mom, h->hp.momentum, h->hp.weight_decay};
     const int grid = (int)std::min<long long>(batches, (long long)h->sm_count * 8);
     const bool bf16 = h->hp.grad_dtype == TA_GRAD_BF16, mom = h->d.mom != nullptr;
-    if (bf16 && mom) ta::k_apply<true, true><<<grid, ta::kThreads, 0, s>>>(aa);
-    else if (bf16) ta::k_apply<true, false><<<grid, ta::kThreads, 0, s>>>(aa);
-    else if (mom) ta::k_apply<false, true><<<grid, ta::kThreads, 0, s>>>(aa);
-    else ta::k_apply<false, false><<<grid, ta::kThreads, 0, s>>>(aa);
+    if (bf16 && mom) launch_after(ta::k_apply<true, true>, (unsigned)grid, 0, s, aa);
+    else if (bf16) launch_after(ta::k_apply<true, false>, (unsigned)grid, 0, s, aa);
+    else if (mom) launch_after(ta::k_apply<false, true>, (unsigned)grid, 0, s, aa);
+    else launch_after(ta::k_apply<false, false>, (unsigned)grid, 0, s, aa);
     ++h->launches;
 }
 
@@ -1051,7 +1066,7 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
     da.has_hz = Hz ? 1u : 0u; da.control = (step % h->hp.t_ctrl) == 0 ? 1u : 0u; da.topk = topk ? 1u : 0u;
     da.step = step;
     da.hist = d.hist; da.sel = d.sel; da.cand_count = d.cand_count; da.seg_k = d.seg_k; da.window = d.window;
-    ta::k_decide<<<h->L, ta::kThreads, 0, s>>>(da);
+    launch_after(ta::k_decide, h->L, 0, s, da);
     ++h->launches;
 
     if (topk) {
@@ -1067,10 +1082,10 @@ static int step_impl(ta_handle *h, float *w, const void *g, const float *Hz, uin
         ta::ApplyArgs aa{d.items, h->n_items, h->n_batches, w, g, c, d.state, d.status, d.mom, h->hp.momentum, h->hp.weight_decay};
         const unsigned blocks = (unsigned)h->L + (unsigned)grid;
         const bool mom = d.mom != nullptr;
-        if (bf16 && mom) ta::k_apply_resolve<true, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-        else if (bf16) ta::k_apply_resolve<true, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-        else if (mom) ta::k_apply_resolve<false, true><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
-        else ta::k_apply_resolve<false, false><<<blocks, ta::kThreads, 0, s>>>(aa, ra, h->L);
+        if (bf16 && mom) launch_after(ta::k_apply_resolve<true, true>, blocks, 0, s, aa, ra, h->L);
+        else if (bf16) launch_after(ta::k_apply_resolve<true, false>, blocks, 0, s, aa, ra, h->L);
+        else if (mom) launch_after(ta::k_apply_resolve<false, true>, blocks, 0, s, aa, ra, h->L);
+        else launch_after(ta::k_apply_resolve<false, false>, blocks, 0, s, aa, ra, h->L);
         ++h->launches;
         if (timed) { cudaEventRecord(ev[3], s); ++h->timed_used; }
         TA_CUDA(h, cudaGetLastError());
