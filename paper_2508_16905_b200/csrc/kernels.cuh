@@ -463,7 +463,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
         // a batch whose items share one layer counts its histogram in shared memory and flushes it once
         bool uniform = false;
         uint32_t batch_layer = 0;
-        if (TOPK) {
+        if (TOPK && !A.redo) {          // (the second sweep counts nothing)
             batch_layer = A.batch_seg[batch];
             uniform = batch_layer != kMixedBatch;
             if (uniform)
@@ -754,7 +754,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             if (lane == 0) A.p_mass[it] = mass;
         }
         }   // item.len != 0
-        if (TOPK) {
+        if (TOPK && !A.redo) {
             __syncthreads();
             if (uniform)
                 for (uint32_t b = threadIdx.x; b < (uint32_t)kHistBins; b += kThreads) {
