@@ -304,23 +304,28 @@ constexpr uint32_t kMixedBatch = 0xFFFFFFFFu;
 
 constexpr uint32_t kStageCap = 384;      // candidates a warp collects in shared memory before it reserves list slots
 
-// Stages this lane's candidates (bit e of `cand` = element e of its vector) in the warp's shared-memory
-// buffer, behind the `running` ones already there.  Whole warp; `running` stays warp-uniform.
-__device__ __forceinline__ void stage_candidates(uint32_t cand, const uint32_t (&ab)[4], uint32_t local0, uint32_t lane,
-                                                 uint32_t &running, uint32_t *sval, uint32_t *sidx)
+// Stages this lane's candidates (bit e of `cand` = element e of its vector) in the warp's shared-memory buffer.
+// A lane with candidates reserves its places on the warp's counter `count` (a shared-memory word); `bound` is a
+// warp-uniform upper bound of that counter, which is all the caller needs to know when to empty the buffer.
+// Whole warp; returns whether anything was staged.  The order of the staged candidates is arbitrary (so is the order
+// of the layer's list).
+__device__ __forceinline__ bool stage_candidates(uint32_t cand, const uint32_t (&ab)[4], uint32_t local0,
+                                                 uint32_t &bound, uint32_t *count, uint32_t *sval, uint32_t *sidx)
 {
-    if (!__any_sync(0xFFFFFFFFu, cand != 0u)) return;
-    const uint32_t below = (1u << lane) - 1u;
+    const uint32_t who = __ballot_sync(0xFFFFFFFFu, cand != 0u);
+    if (who == 0u) return false;
+    bound += 4u * (uint32_t)__popc(who);
+    if (cand != 0u) {
+        uint32_t pos = atomicAdd(count, (uint32_t)__popc(cand));
 #pragma unroll
-    for (uint32_t e = 0; e < 4; ++e) {
-        const uint32_t who = __ballot_sync(0xFFFFFFFFu, (cand >> e) & 1u);
-        if ((cand >> e) & 1u) {
-            const uint32_t pos = running + (uint32_t)__popc(who & below);
-            sval[pos] = ab[e];
-            sidx[pos] = local0 + e;
-        }
-        running += (uint32_t)__popc(who);
+        for (uint32_t e = 0; e < 4; ++e)
+            if ((cand >> e) & 1u) {
+                sval[pos] = ab[e];
+                sidx[pos] = local0 + e;
+                ++pos;
+            }
     }
+    return true;
 }
 
 // 8 lanes make one 32-bit mask word out of their 4-bit pieces.
@@ -399,16 +404,19 @@ template <int P, bool TOPK> struct SweepAcc {
     double pivot = 0.0;     // subtracted from every gradient value before it is summed
     double s1 = 0.0, s2 = 0.0, sa = 0.0;
     float sa_row = 0.f;     // |S| of the current row (four values), folded into sa by end_row()
-    uint32_t amax = 0u, amin = 0xFFFFFFFFu, gmax = 0u;
+    uint32_t amax = 0u, amin = 0xFFFFFFFFu;   // amin is kept only without top-k (it is the dense threshold)
 
     __device__ __forceinline__ void end_row() { sa += (double)sa_row; sa_row = 0.f; }
 
-    // one element: gradient value gv, probe products hv[p], sign words sel[p], bit position pos
+    // A non-finite gradient value (or pivot) makes s2 non-finite, and finite values cannot: |x| < 2^129, so
+    // the sum of 2^64 squares still fits a double.  That is the screen of the gradients; no maximum is kept.
+    static __device__ __forceinline__ bool gradients_suspect(double s2_total) { return !(s2_total < (double)INFINITY); }
+
+    // one element: gradient value gv, probe products hv[p], sign words of the row sel[p] with the sign bit of the
+    // lane's element 0 moved to bit 28 (element e: bit 28 + e), e = 0..3
     __device__ __forceinline__ uint32_t element(float gv, const float (&hv)[P > 0 ? P : 1],
-                                                const uint32_t (&sel)[P > 0 ? P : 1], uint32_t pos)
+                                                const uint32_t (&sel)[P > 0 ? P : 1], uint32_t e)
     {
-        const uint32_t gb = __float_as_uint(gv) & 0x7FFFFFFFu;
-        gmax = max(gmax, gb);
         const double x = (double)gv - pivot;
         s1 += x;
         s2 = fma(x, x, s2);
@@ -420,13 +428,13 @@ template <int P, bool TOPK> struct SweepAcc {
 #pragma unroll
             for (int p = 0; p < P; ++p) {
                 const uint32_t hb = __float_as_uint(hv[p]);
-                t[p] = __uint_as_float(hb ^ (((sel[p] >> pos) & 1u) << 31));
+                t[p] = __uint_as_float(hb ^ ((sel[p] << (3u - e)) & 0x80000000u));
             }
             ab = __float_as_uint(pairwise<P>(t)) & 0x7FFFFFFFu;
         }
         if (P > 0) {
             amax = max(amax, ab);
-            amin = min(amin, ab);
+            if (!TOPK) amin = min(amin, ab);
             if (TOPK) sa_row += __uint_as_float(ab);
         }
         return ab;
@@ -446,10 +454,12 @@ struct ItemSums {
 // RING > 0: full rows travel through a ring of RING rows per warp in shared memory (sh_ring, [kWarps][RING][1 + P] rows
 // of 32 x 16 bytes), filled by asynchronous copies that run ahead of the arithmetic: a warp then has loads in flight
 // all the time, not only between two bursts, which is what the multi-probe sweeps (many instructions per byte) need.
-template <int P, bool BF16, bool TOPK, bool APPLY, int ROWS = 0, int RING = 0, typename Store>
+// HIST (top-k) says at compile time where the batch counts its level-1 histogram, which spares the row loop the
+// tests: 0 nowhere (the second sweep), 1 in shared memory (all items in one layer), 2 in the layers' own histograms.
+template <int P, bool BF16, bool TOPK, bool APPLY, int ROWS = 0, int RING = 0, int HIST = 1, typename Store>
 __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, uint32_t *sh_hist, const Store &store,
                                             const SinglePass &sp = SinglePass{nullptr, nullptr, nullptr, 0.f},
-                                            uint32_t *sh_stage = nullptr /* TOPK: [kWarps][2][kStageCap] */,
+                                            uint32_t *sh_stage = nullptr /* TOPK: [kWarps][2][kStageCap], then [kWarps] counters */,
                                             float4 *sh_ring = nullptr)
 {
     static_assert(!(RING > 0 && (APPLY || P == 0)), "the ring is for sweeps with probe products");
@@ -461,11 +471,10 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
     {
         const uint32_t it = batch * kWarps + warp;
         // a batch whose items share one layer counts its histogram in shared memory and flushes it once
-        bool uniform = false;
+        constexpr bool uniform = TOPK && HIST == 1, redo = TOPK && HIST == 0;
         uint32_t batch_layer = 0;
-        if (TOPK && !A.redo) {          // (the second sweep counts nothing)
+        if (TOPK && !redo) {          // (the second sweep counts nothing)
             batch_layer = A.batch_seg[batch];
-            uniform = batch_layer != kMixedBatch;
             if (uniform)
                 for (uint32_t b = threadIdx.x; b < (uint32_t)kHistBins; b += kThreads) sh_hist[b] = 0u;
             __syncthreads();
@@ -478,7 +487,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
         // top-k: the window of level-1 bins this pass works with, and whether it touches the mask at all
         uint32_t win_lo = 1u, win_hi = 0u;
         if (TOPK && item.len != 0u) {
-            if (A.redo) {
+            if (redo) {
                 const SelectState ss = A.sel[item.seg];
                 if (ss.valid) item.len = 0u;                   // the first pass got this layer right
                 win_lo = win_hi = ss.prefix;
@@ -488,6 +497,9 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             }
         }
         const bool masking = TOPK && win_lo <= win_hi;
+        // the same window on the bit patterns: above it from thr_hi on (2^31 when the window ends at the last bin: no
+        // pattern of a magnitude reaches that), inside it from thr_lo on
+        const uint32_t thr_lo = win_lo << 20, thr_hi = (win_hi + 1u) << 20;
         if (item.len != 0u) {
         const uint64_t begin = item.begin, end = begin + item.len;
         const uint64_t row_first = begin >> 7, row_last = (end - 1) >> 7;
@@ -501,27 +513,35 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             code = sp.state[item.seg].code;
         }
         auto hist_add = [&](uint32_t ab) {
-            if (A.redo) return;
+            if (redo) return;
             if (uniform) atomicAdd(&sh_hist[ab >> 20], 1u);
             else atomicAdd(A.hist + (uint64_t)item.seg * kHistBins + (ab >> 20), 1u);
         };
         // top-k: mask bits above the window, candidates inside it
         const uint64_t seg_b = TOPK ? A.seg_off[item.seg] : 0ull;
-        uint32_t *mask = TOPK ? A.mask2 + (size_t)(A.redo ? A.status->mask_cur : 1u - A.status->mask_cur) * A.mask_words : nullptr;
+        uint32_t *mask = TOPK ? A.mask2 + (size_t)(redo ? A.status->mask_cur : 1u - A.status->mask_cur) * A.mask_words : nullptr;
         uint32_t *sval = TOPK ? sh_stage + (size_t)warp * 2u * kStageCap : nullptr, *sidx = TOPK ? sval + kStageCap : nullptr;
-        uint32_t staged = 0u;
+        uint32_t *scount = TOPK ? sh_stage + (size_t)kWarps * 2u * kStageCap + warp : nullptr;      // candidates staged by this warp
+        uint32_t staged = 0u;                                   // upper bound of *scount, warp-uniform
         double mass = 0.0;
+        if (TOPK) {
+            if (lane == 0) *scount = 0u;
+            __syncwarp();
+        }
         // moves the staged candidates to the layer's list: one slot reservation for all of them
         auto flush = [&]() {
             if (staged == 0u) return;
-            uint32_t base = 0;
-            if (lane == 0) base = atomicAdd(A.cand_count + item.seg, staged);
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
             __syncwarp();
-            for (uint32_t j = lane; j < staged; j += 32) {
+            const uint32_t n = *scount;
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(A.cand_count + item.seg, n);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            for (uint32_t j = lane; j < n; j += 32) {
                 A.cand_val[seg_b + base + j] = sval[j];
                 A.cand_idx[seg_b + base + j] = sidx[j];
             }
+            __syncwarp();
+            if (lane == 0) *scount = 0u;
             __syncwarp();
             staged = 0u;
         };
@@ -531,15 +551,27 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             float above = 0.f;
 #pragma unroll
             for (uint32_t e = 0; e < 4; ++e) {
-                const uint32_t bin = ab[e] >> 20;
-                if ((inside >> e) & 1u) {
-                    if (bin > win_hi) { nib |= 1u << e; above += __uint_as_float(ab[e]); }
-                    else if (bin >= win_lo) cand |= 1u << e;
-                }
+                const bool over = ab[e] >= thr_hi, reach = ab[e] >= thr_lo;       // selects, no branches
+                nib |= over ? 1u << e : 0u;
+                cand |= reach ? 1u << e : 0u;
+                above += over ? __uint_as_float(ab[e]) : 0.f;
+            }
+            nib &= inside;
+            cand &= inside & ~nib;
+            if (!whole) {         // elements outside the item carry no value, but say so where it costs nothing
+                above = 0.f;
+#pragma unroll
+                for (uint32_t e = 0; e < 4; ++e) above += (nib >> e) & 1u ? __uint_as_float(ab[e]) : 0.f;
             }
             mass += (double)above;
             if (staged + 128u > kStageCap) flush();
-            stage_candidates(cand, ab, (uint32_t)(row * 128ull - seg_b) + lane * 4u, lane, staged, sval, sidx);
+            stage_candidates(cand, ab, (uint32_t)(row * 128ull - seg_b) + lane * 4u, staged, scount, sval, sidx);
+            if (whole) {
+                // two lanes make one byte of the row's 16 mask bytes (little-endian words: byte j = bits 8j .. 8j+7)
+                const uint32_t pair = nib | (__shfl_xor_sync(0xFFFFFFFFu, nib, 1) << 4);
+                if ((lane & 1u) == 0u) reinterpret_cast<uint8_t *>(mask)[row * 16ull + (lane >> 1)] = (uint8_t)pair;
+                return;
+            }
             const uint32_t word = gather_word(nib, lane);
             if ((lane & 7u) == 0u) {
                 const uint64_t w0 = row * 128ull + (lane >> 3) * 32ull;     // first element of this word
@@ -576,7 +608,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             const uint32_t k = (uint32_t)(row & 31u);
             uint32_t sel[PP];
 #pragma unroll
-            for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
+            for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) << (28u - (k & 7u) * 4u) : 0u;
             const uint64_t i0 = row * 128ull + lane * 4u;
             uint32_t abs4[4] = {0u, 0u, 0u, 0u}, inside = 0u;
 #pragma unroll
@@ -587,7 +619,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
 #pragma unroll
                     for (int p = 0; p < PP; ++p) hv[p] = (P > 0) ? __ldcs(A.hz + (uint64_t)p * A.n_total + i) : 0.f;
                     const float gv = GradVec<BF16>::load1(A.g, i);
-                    const uint32_t ab = acc.element(gv, hv, sel, (k & 7u) * 4u + e);
+                    const uint32_t ab = acc.element(gv, hv, sel, e);
                     abs4[e] = ab;
                     inside |= 1u << e;
                     if (APPLY) {
@@ -604,16 +636,40 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             }
         };
 
+        // top-k bookkeeping of one full row: level-1 histogram, mask bits, candidates
+        auto count_row = [&](const uint32_t (&abs4)[4]) {
+            // exact zeros (pruned or untouched weights) would all hit one counter: the warp counts them together
+            uint32_t zeros = 0u;
+#pragma unroll
+            for (uint32_t e = 0; e < 4; ++e) {
+                zeros += (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, abs4[e] == 0u));
+                if (abs4[e] != 0u) hist_add(abs4[e]);
+            }
+            if (lane == 0 && !redo) {
+                if (uniform) atomicAdd(&sh_hist[0], zeros);
+                else atomicAdd(A.hist + (uint64_t)item.seg * kHistBins, zeros);
+            }
+        };
+        auto book_row = [&](uint64_t row, const uint32_t (&abs4)[4]) {
+            const uint32_t least = min(min(abs4[0], abs4[1]), min(abs4[2], abs4[3]));
+            if (__any_sync(0xFFFFFFFFu, least == 0u)) {
+                count_row(abs4);
+            } else {
+#pragma unroll
+                for (uint32_t e = 0; e < 4; ++e) hist_add(abs4[e]);
+            }
+            if (masking) mask_row(row, abs4, 0xFu, true);
+        };
         auto full_rows = [&](uint64_t row, RowData<P> (&rd)[U], int count) {
+            uint32_t abs_all[U][4];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (u < count) {
                     const uint32_t k = (uint32_t)((row + u) & 31u);
                     uint32_t sel[PP];
 #pragma unroll
-                    for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
+                    for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) << (28u - (k & 7u) * 4u) : 0u;
                     const float gv[4] = {rd[u].g.x, rd[u].g.y, rd[u].g.z, rd[u].g.w};
-                    uint32_t abs4[4];
 #pragma unroll
                     for (uint32_t e = 0; e < 4; ++e) {
                         float hv[PP];
@@ -622,26 +678,16 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
                             const float4 h = rd[u].hz[p];
                             hv[p] = e == 0 ? h.x : (e == 1 ? h.y : (e == 2 ? h.z : h.w));
                         }
-                        const uint32_t ab = acc.element(gv[e], hv, sel, (k & 7u) * 4u + e);
-                        abs4[e] = ab;
+                        abs_all[u][e] = acc.element(gv[e], hv, sel, e);
                     }
-                    if (TOPK) {
-                        // exact zeros (pruned or untouched weights) would all hit one counter: the warp counts them together
-                        uint32_t zeros = 0u;
-#pragma unroll
-                        for (uint32_t e = 0; e < 4; ++e) {
-                            zeros += (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, abs4[e] == 0u));
-                            if (abs4[e] != 0u) hist_add(abs4[e]);
-                        }
-                        if (lane == 0 && zeros != 0u && !A.redo) {
-                            if (uniform) atomicAdd(&sh_hist[0], zeros);
-                            else atomicAdd(A.hist + (uint64_t)item.seg * kHistBins, zeros);
-                        }
-                        acc.end_row();
-                        if (masking) mask_row(row + u, abs4, 0xFu, true);
-                    }
+                    if (TOPK) acc.end_row();
                     if (APPLY) update_store4<true>(sp.w, sp.c, (row + u) * 128ull + lane * 4u, rd[u].w, rd[u].g, neg_eta, code);
                 }
+            }
+            if constexpr (TOPK) {
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (u < count) book_row(row + u, abs_all[u]);
             }
         };
 
@@ -683,20 +729,23 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
 #pragma unroll
             for (int r = 0; r < RING; ++r) issue(full_lo + r, r);
             int slot = 0;
-            for (uint64_t row = full_lo; row < full_hi; ++row) {
-                cp_async_wait_group<RING - 1>();
-                refresh(row);
-                const float4 *src = mine + (size_t)slot * (1 + PP) * 32u;
-                RowData<P> rd[1];
+            auto take = [&](int sl, RowData<P> &r) {
+                const float4 *src = mine + (size_t)sl * (1 + PP) * 32u;
                 if (BF16) {
                     const uint2 v = *reinterpret_cast<const uint2 *>(src);
-                    rd[0].g = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
-                                          __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+                    r.g = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
+                                      __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
                 } else {
-                    rd[0].g = src[0];
+                    r.g = src[0];
                 }
 #pragma unroll
-                for (int p = 0; p < PP; ++p) rd[0].hz[p] = src[(size_t)(1 + p) * 32u];
+                for (int p = 0; p < PP; ++p) r.hz[p] = src[(size_t)(1 + p) * 32u];
+            };
+            for (uint64_t row = full_lo; row < full_hi; ++row) {
+                RowData<P> rd[U];
+                cp_async_wait_group<RING - 1>();
+                refresh(row);
+                take(slot, rd[0]);
                 issue(row + RING, slot);          // the slot is free again: the values are in registers
                 full_rows(row, rd, 1);
                 slot = slot + 1 == RING ? 0 : slot + 1;
@@ -733,12 +782,11 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
         const double sa = TOPK ? warp_sum(acc.sa) : 0.0;
         const uint32_t amax = __reduce_max_sync(0xFFFFFFFFu, acc.amax);
         const uint32_t amin = __reduce_min_sync(0xFFFFFFFFu, acc.amin);
-        const uint32_t gmax = __reduce_max_sync(0xFFFFFFFFu, acc.gmax);
         // a non-finite Hz value always makes its probe sum non-finite, so max|S| flags it (a sum of finite values
         // that overflows also lands here; the exact recount below then finds nothing)
         const uint32_t hmax = amax;
         uint32_t bad = 0;
-        if (gmax >= kNonFiniteBits || (P > 0 && hmax >= kNonFiniteBits)) {
+        if (SweepAcc<P, TOPK>::gradients_suspect(s2) || (P > 0 && hmax >= kNonFiniteBits)) {
             // rare: count the non-finite inputs of this item exactly
             for (uint64_t i = begin + lane; i < end; i += 32) {
                 if ((__float_as_uint(GradVec<BF16>::load1(A.g, i)) & 0x7FFFFFFFu) >= kNonFiniteBits) ++bad;
@@ -754,7 +802,7 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             if (lane == 0) A.p_mass[it] = mass;
         }
         }   // item.len != 0
-        if (TOPK && !A.redo) {
+        if (TOPK && !redo) {
             __syncthreads();
             if (uniform)
                 for (uint32_t b = threadIdx.x; b < (uint32_t)kHistBins; b += kThreads) {
@@ -775,7 +823,7 @@ template <int P, bool BF16, bool TOPK>
 __global__ void __launch_bounds__(kThreads, ((P == 4 || TOPK) && P <= 4 ? 2 : 1)) k_sweep(const SweepArgs A)
 {
     __shared__ uint32_t sh_hist[TOPK ? kHistBins : 1];
-    __shared__ uint32_t sh_stage[TOPK ? kWarps * 2 * kStageCap : 1];
+    __shared__ uint32_t sh_stage[TOPK ? kWarps * 2 * kStageCap + kWarps : 1];     // + one counter per warp
     extern __shared__ __align__(16) float4 sh_ring[];          // TOPK: kWarps * kSweepRing<P> rows of (1 + P) x 512 bytes
     grid_dependency_wait();         // launched ahead of time: the kernel before this one is complete from here on
     grid_dependency_release();
@@ -788,7 +836,14 @@ __global__ void __launch_bounds__(kThreads, ((P == 4 || TOPK) && P <= 4 ? 2 : 1)
         if (P > 0) { A.p_amax[it] = r.amax; A.p_amin[it] = r.amin; }
         if (TOPK) A.p_sa[it] = r.sa;
     };
-    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) sweep_batch<P, BF16, TOPK, false, 0, (TOPK ? sweep_ring_rows(P) : 0)>(A, batch, sh_hist, store, SinglePass{nullptr, nullptr, nullptr, 0.f}, sh_stage, sh_ring);
+    constexpr int R = TOPK ? sweep_ring_rows(P) : 0;
+    const SinglePass none{nullptr, nullptr, nullptr, 0.f};
+    for (uint32_t batch = blockIdx.x; batch < A.n_batches; batch += gridDim.x) {
+        if (!TOPK) sweep_batch<P, BF16, TOPK, false, 0, R>(A, batch, sh_hist, store, none, sh_stage, sh_ring);
+        else if (A.redo) sweep_batch<P, BF16, TOPK, false, 0, R, 0>(A, batch, sh_hist, store, none, sh_stage, sh_ring);
+        else if (A.batch_seg[batch] != kMixedBatch) sweep_batch<P, BF16, TOPK, false, 0, R, 1>(A, batch, sh_hist, store, none, sh_stage, sh_ring);
+        else sweep_batch<P, BF16, TOPK, false, 0, R, 2>(A, batch, sh_hist, store, none, sh_stage, sh_ring);
+    }
 }
 
 // ------------------------------------------------------------------ decisions
@@ -1436,10 +1491,9 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
             const double s1 = warp_sum(acc.s1), s2 = warp_sum(acc.s2);
             const uint32_t amax = __reduce_max_sync(0xFFFFFFFFu, acc.amax);
             const uint32_t amin = __reduce_min_sync(0xFFFFFFFFu, acc.amin);
-            const uint32_t gmax = __reduce_max_sync(0xFFFFFFFFu, acc.gmax);
             uint32_t bad = 0u;
             // a non-finite Hz value always makes its probe sum non-finite, so max|S| flags it
-            if (gmax >= kNonFiniteBits || (P > 0 && amax >= kNonFiniteBits)) {
+            if (SweepAcc<P, false>::gradients_suspect(s2) || (P > 0 && amax >= kNonFiniteBits)) {
                 // rare: count the non-finite inputs of this run exactly
                 const Item item = A.runs[run_lo + run];
                 for (uint64_t i = item.begin + lane; i < item.begin + item.len; i += 32) {
@@ -1513,7 +1567,7 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
                         }
                     }
 #pragma unroll
-                    for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) : 0u;
+                    for (int p = 0; p < PP; ++p) sel[p] = (P > 1) ? pick_word(X[p], k >> 3) << (28u - (k & 7u) * 4u) : 0u;
 #pragma unroll
                     for (uint32_t e = 0; e < 4; ++e) {
                         if (e >= e_lo && e < e_hi) {
@@ -1523,7 +1577,7 @@ __global__ void __launch_bounds__(kThreads, (P <= 1 ? TA_FUSED_MIN_BLOCKS : (P <
                                 const float4 h = rd[u].hz[p];
                                 hv[p] = e == 0 ? h.x : (e == 1 ? h.y : (e == 2 ? h.z : h.w));
                             }
-                            acc.element(gv[e], hv, sel, (k & 7u) * 4u + e);
+                            acc.element(gv[e], hv, sel, e);
                         }
                     }
                     if (s0 + u < A.cap_g && e_hi > e_lo) sh_g[(s0 + u) * 32u + lane] = rd[u].g;

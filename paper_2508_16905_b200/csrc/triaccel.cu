@@ -72,6 +72,7 @@ struct ta_handle {
     uint32_t n_items = 0, n_batches = 0, item_elems = 0;
     uint64_t mask_words = 0;
     bool topk = false;
+    bool ring_asked = false;          // the top-k sweep's shared-memory ring has been allowed on this device
     bool stepped = false;
     uint64_t last_step = 0;
     uint64_t launches = 0;
@@ -206,14 +207,14 @@ template <int P, bool BF16, bool TOPK> void launch_sweep(ta_handle *h, const ta:
 {
     // the top-k sweeps stage their rows in a ring of shared memory (beyond the 48 KB a launch gets without asking)
     const size_t ring = TOPK ? ta::sweep_ring_bytes(P) : 0;
-    if (TOPK) {
-        static bool asked = false;          // per instantiation
-        if (!asked) {
-            cudaFuncSetAttribute(ta::k_sweep<P, BF16, TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring);
-            asked = true;
-        }
+    if (TOPK && !h->ring_asked) {           // per device and kernel; a handle has one of each
+        cudaFuncSetAttribute(ta::k_sweep<P, BF16, TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring);
+        h->ring_asked = true;
     }
-    launch_after(ta::k_sweep<P, BF16, TOPK>, (unsigned)grid_for(h), ring, s, a);
+    // the second sweep of a top-k step usually finds nothing to repeat: one resident wave of blocks, which walk the
+    // batches in a loop, starts (and ends) faster than a block per batch and is as fast when there is work
+    const unsigned grid = TOPK && a.redo ? (unsigned)std::min<long long>(grid_for(h), (long long)h->sm_count * 2) : (unsigned)grid_for(h);
+    launch_after(ta::k_sweep<P, BF16, TOPK>, grid, ring, s, a);
     ++h->launches;
 }
 
