@@ -196,6 +196,30 @@ __device__ __forceinline__ void cp_async8_stream(void *smem, const void *gmem)
     const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(gmem) : "memory");
 }
+// The same with a say in what L2 keeps: `policy` from createpolicy (evict_first for data that is read once,
+// evict_last for data that a later kernel of the step reads again).
+__device__ __forceinline__ void cp_async16_hint(void *smem, const void *gmem, uint64_t policy)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(s), "l"(gmem), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void cp_async8_hint(void *smem, const void *gmem, uint64_t policy)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global.L2::cache_hint [%0], [%1], 8, %2;" ::"r"(s), "l"(gmem), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ uint64_t l2_evict_last_policy()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
 __device__ __forceinline__ void cp_async_commit_group() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -715,14 +739,16 @@ __device__ __forceinline__ void sweep_batch(const SweepArgs &A, uint32_t batch, 
             // this lane's 16-byte pieces of RING rows are on their way while it works on the oldest one; a lane reads
             // back only what it copied itself, so the wait for its own copies is all the ordering needed
             float4 *mine = sh_ring + (size_t)warp * RING * (1 + PP) * 32u + lane;
+            const uint64_t keep = l2_evict_last_policy(), once = l2_evict_first_policy();
             auto issue = [&](uint64_t row, int slot) {
                 if (row < full_hi) {
                     const uint64_t i0 = row * 128ull + lane * 4u;
                     float4 *dst = mine + (size_t)slot * (1 + PP) * 32u;
-                    if (BF16) cp_async8_stream(dst, static_cast<const uint16_t *>(A.g) + i0);
-                    else cp_async16_stream(dst, static_cast<const float *>(A.g) + i0);
+                    // the update reads the gradient again, nothing reads the probe products again
+                    if (BF16) cp_async8_hint(dst, static_cast<const uint16_t *>(A.g) + i0, keep);
+                    else cp_async16_hint(dst, static_cast<const float *>(A.g) + i0, keep);
 #pragma unroll
-                    for (int p = 0; p < PP; ++p) cp_async16_stream(dst + (size_t)(1 + p) * 32u, A.hz + (uint64_t)p * A.n_total + i0);
+                    for (int p = 0; p < PP; ++p) cp_async16_hint(dst + (size_t)(1 + p) * 32u, A.hz + (uint64_t)p * A.n_total + i0, once);
                 }
                 cp_async_commit_group();          // one group per row, empty behind the last row, so that the count below holds
             };
@@ -1361,19 +1387,6 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 // All groups of copies but the newest one have arrived.
 __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
-// Data that passes through L2 once is the first to leave it again; the plan, read by every launch, the last.
-__device__ __forceinline__ uint64_t l2_evict_first_policy()
-{
-    uint64_t policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    return policy;
-}
-__device__ __forceinline__ uint64_t l2_evict_last_policy()
-{
-    uint64_t policy;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
-    return policy;
-}
 __device__ __forceinline__ uint4 ld_plan(const void *p, uint64_t policy)
 {
     uint4 v;
