@@ -2145,7 +2145,11 @@ __global__ void __launch_bounds__(kThreads) k_apply_resolve(const ApplyArgs A, c
     const LayerState *state = A.state;
     // eta and code were fixed by k_decide; resolve blocks write other fields (threshold, mass) of the same records
     auto decision = [state](uint32_t seg, float &eta, uint32_t &code) { eta = state[seg].eta; code = state[seg].code; };
-    for (uint32_t batch = blockIdx.x - n_layers; batch < A.n_batches; batch += gridDim.x - n_layers) apply_batch<BF16, MOM, TA_APPLY_STREAM_W_STORE != 0>(A, batch, decision);
+    // the new weights are stored with the streaming hint: what is worth keeping in L2 is the gradient that the sweep
+    // has just read (measured on the ResNet-50 mix: update 49.6 -> 45.9 us; walking the batches from the end, as
+    // k_apply does, was slower here)
+    for (uint32_t batch = blockIdx.x - n_layers; batch < A.n_batches; batch += gridDim.x - n_layers)
+        apply_batch<BF16, MOM, true>(A, batch, decision);
 }
 
 }  // namespace ta
