@@ -166,11 +166,15 @@ def test_tie_breaks_lower_index_first():
     D = np.full(n_total, 0.25, dtype=np.float32)
     D[70010:70010 + 5000:2] = 0.75
     g = torch.zeros(n_total, device="cuda")
-    run.step(1, g, oracle_hz(D, 2, 4, 1), 4)
-    m = ta.ta_masks_to_host(run.h)
     idx = np.arange(3, 3 + 70000)
-    bits = (m[idx >> 5] >> (idx & 31).astype(np.uint32)) & 1
-    assert np.array_equal(bits, (np.arange(70000) < 17500).astype(np.uint32))
+    # step 1 has no window yet (every layer is swept a second time with the exact bin); steps 2 and 3 select inside
+    # the window, where every element of layer 0 is a candidate: the warps' candidate stages fill and empty all the time
+    for t in (1, 2, 3):
+        run.step(t, g, oracle_hz(D, 2, 4, t), 4)
+        m = ta.ta_masks_to_host(run.h)
+        bits = (m[idx >> 5] >> (idx & 31).astype(np.uint32)) & 1
+        assert np.array_equal(bits, (np.arange(70000) < 17500).astype(np.uint32))
+    assert ta.ta_launch_count(run.h) == 3 * 4
 
 
 @pytest.mark.parametrize("P", [1, 4])
