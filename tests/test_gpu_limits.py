@@ -122,3 +122,45 @@ def test_random_tables(seed):
         if grad_dtype == "bf16":
             g_dev = g_dev.to(torch.bfloat16)
         run.step(t, g_dev, oracle_hz(D, P, seed, t) if t != 2 else None, seed)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_tables_with_large_layers_and_drifting_curvature(seed):
+    # layers up to 700,000 elements; curvature that stays, drifts by a few per cent, is absent on a step and jumps by
+    # a factor of eight; inputs with few distinct values, with exact zeros (pruned weights) or with every value equal:
+    # the sweep's window of bins, its candidate lists, the second sweep and the resolve step against the oracle
+    rng = np.random.default_rng(5000 + seed)
+    L = int(rng.integers(1, 12))
+    lengths = []
+    for _ in range(L):
+        r = rng.random()
+        lengths.append(int(rng.integers(1, 300)) if r < 0.3 else int(rng.integers(300, 30000)) if r < 0.7 else int(rng.integers(30000, 700000)))
+    table, off = [], int(rng.integers(0, 9))
+    for n in lengths:
+        off += int(rng.integers(0, 4)) * int(rng.random() < 0.5)
+        table.append((off, n))
+        off += n
+    n_total = (off + int(rng.integers(0, 9)) + 3) // 4 * 4
+    P = int(rng.choice([1, 2, 4, 8]))
+    ppm = int(rng.choice([1000, 100000, 500000, 900000])) if rng.random() < 0.8 else 1000000
+    grad_dtype = "bf16" if rng.random() < 0.4 else "f32"
+    hp = dict(beta=0.9, tau_low=3e-7, tau_high=3e-6, tau_curv=0.5, alpha=1.0, eta0=0.05, topk_ppm=ppm, num_probes=P,
+              t_ctrl=int(rng.choice([1, 2])), grad_dtype=grad_dtype)
+    run = ParityRun(table, n_total, hp, torch.from_numpy((rng.standard_normal(n_total) * 0.05).astype(np.float32)))
+    D0 = np.exp(rng.uniform(np.log(1e-4), 0.5, n_total)).astype(np.float32)
+    mode = int(rng.integers(0, 4))
+    if mode == 1:
+        D0 = np.round(D0 * 8) / 8 + np.float32(0.125)
+    elif mode == 2:
+        D0[rng.random(n_total) < 0.6] = 0.0
+    elif mode == 3:
+        D0[:] = np.float32(0.5)
+    sigma = 10.0 ** rng.uniform(-4.5, -2.0, L)
+    for t, f in enumerate([1.0, 1.02, None, 0.97, 8.0, 1.0], start=1):
+        g = np.zeros(n_total, dtype=np.float32)
+        for (o, n), s in zip(table, sigma):
+            g[o:o + n] = rng.standard_normal(n) * s
+        g_dev = torch.from_numpy(g).cuda()
+        if grad_dtype == "bf16":
+            g_dev = g_dev.to(torch.bfloat16)
+        run.step(t, g_dev, oracle_hz(D0 * np.float32(f), P, seed, t) if f is not None else None, seed)
