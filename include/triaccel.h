@@ -348,7 +348,7 @@ int ta_plan_one_launch(const ta_segment *table, uint32_t L, uint32_t warps, ta_r
  * no GPU needed).  Every task covers one batch: up to 14336 consecutive elements of one layer.  With
  * with_decisions != 0, the two queues of a step that takes decisions (Sec. 3.4), one after the other: the sweep tasks
  * (TA_TASK_SWEEP, statistics) in buffer order, then the update tasks (TA_TASK_APPLY) layer by layer, within a layer
- * in buffer order.  Blocks draw from both queues; an update task is handed out once its layer is decided, and
+ * the last batch first.  Blocks draw from both queues; an update task is handed out once its layer is decided, and
  * until then the block goes on sweeping.  Otherwise the queue of a step between decisions, one single-pass task
  * (TA_TASK_BOTH) per batch.  Writes at most cap tasks; *n_tasks is their number (TA_ERR_ARG if cap is smaller).
  * Table rules as for ta_create.

@@ -12,9 +12,8 @@
 //   both   batch b   steps without decisions (step % T_ctrl != 0, Sec. 3.4): the step size and code of every layer are
 //                    known beforehand, so statistics, update and cast run in a single pass over the data
 //
-// A step with decisions has two queues, sweep tasks in buffer order and apply tasks layer by layer (within a layer in
-// buffer order too: measured faster than the last batch first, although that order finds more of the gradient still in
-// L2: both streams then walk the memory in the same direction).  Blocks draw tickets from both; an apply
+// A step with decisions has two queues, sweep tasks in buffer order and apply tasks layer by layer (within a layer the
+// last batch first: the rows swept last are the ones most surely still in L2).  Blocks draw tickets from both; an apply
 // task is handed out only once its layer's decisions are published, and until then the block keeps sweeping, so a
 // layer is updated as soon as it is decided and nobody ever waits for anybody: a block polls, it never blocks, and the
 // launch needs no co-residency.  A step without decisions has only the queue of single-pass tasks.

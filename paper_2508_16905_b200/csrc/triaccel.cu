@@ -380,7 +380,7 @@ RunPlan plan_runs(const ta_segment *table, uint32_t L, uint64_t max_warps)
 
 // The plan of the layer-pipelined pass: batches of kPipeCells cells of kPipeItemElems elements cut on a global grid,
 // every batch inside one layer, and the task queues.  A step with decisions: the sweep tasks in buffer order, and the
-// apply tasks layer by layer, within a layer in buffer order.  A step without decisions: one single-pass task
+// apply tasks layer by layer, within a layer the last batch first.  A step without decisions: one single-pass task
 // per batch, in buffer order.
 struct PipePlan {
     std::vector<uint32_t> batch_lo;
@@ -417,7 +417,7 @@ PipePlan plan_pipe(const ta_segment *table, uint32_t L)
         pl.sweep.push_back(task_of(b, ta::kTaskSweep));
     }
     for (uint32_t l = 0; l < L; ++l)
-        for (uint32_t b = pl.batch_lo[l]; b < pl.batch_lo[l + 1]; ++b) pl.apply.push_back(task_of(b, ta::kTaskApply));
+        for (uint32_t b = pl.batch_lo[l + 1]; b-- > pl.batch_lo[l];) pl.apply.push_back(task_of(b, ta::kTaskApply));
     return pl;
 }
 

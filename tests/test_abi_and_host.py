@@ -163,11 +163,11 @@ def test_pipeline_queues_cover_every_layer_once():
         sweeps, applies = both[:len(hold)], both[len(hold):]
         assert all(k == 0 for k, _, _, _ in sweeps) and all(k == 1 for k, _, _, _ in applies)
         assert [x[1:] for x in sweeps] == [x[1:] for x in hold]
-        # update tasks: layer by layer, a layer's batches in buffer order
+        # update tasks: layer by layer, a layer's last batch first
         assert [l for _, l, _, _ in applies] == sorted(l for _, l, _, _ in applies)
         for l in range(len(table)):
             mine = [x[1:] for x in applies if x[1] == l]
-            assert mine == [x[1:] for x in sweeps if x[1] == l]
+            assert mine == [x[1:] for x in sweeps if x[1] == l][::-1]
 
 
 def test_replica_bookkeeping_world_size_2_gloo(tmp_path):
