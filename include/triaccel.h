@@ -344,6 +344,20 @@ int ta_plan_one_launch(const ta_segment *table, uint32_t L, uint32_t warps, ta_r
                        uint32_t *n_runs, uint32_t *warps_used, uint32_t *max_rows);
 
 /*
+ * The work items of the multi-kernel pass (models too large for the one-launch path, top-k masks, momentum), for
+ * inspection (host only, no GPU needed).  Every layer is cut on a global grid of *item_elems elements (512 ... 16384,
+ * chosen from the parameter count so that every warp slot of a GPU with sm_count SMs gets several items); one warp
+ * handles one item, eight consecutive items make the batch of one block.  topk != 0: a layer of at least eight items
+ * starts on a batch boundary (empty padding items, length 0, before it), so that its batches hold one layer only and
+ * count the histogram of Sec. 3.2's selection in shared memory.  Writes the items in buffer order to
+ * out[0 .. *n_items) (at most cap; TA_ERR_ARG if there are more): `warp` is the item's place in its batch, `reserved`
+ * is 1 when all items of that batch lie in one layer.  ta_create builds the same plan with the device's SM count.
+ * Table rules as for ta_create.
+ */
+int ta_plan_items(const ta_segment *table, uint32_t L, uint32_t sm_count, uint32_t topk, ta_run *out, uint64_t cap,
+                  uint64_t *n_items, uint32_t *item_elems);
+
+/*
  * The task queues of the pipelined pass (TA_FLAG_INPUTS_FINITE on a large dense model), for inspection (host only,
  * no GPU needed).  Every task covers one batch: up to 14336 consecutive elements of one layer.  With
  * with_decisions != 0, the two queues of a step that takes decisions (Sec. 3.4), one after the other: the sweep tasks

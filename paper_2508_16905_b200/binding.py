@@ -22,7 +22,7 @@ EXPORTS = ["ta_create", "ta_destroy", "ta_step", "ta_step_host", "ta_set_lr", "t
            "ta_precision_codes", "ta_masks", "ta_launch_count", "ta_last_error", "ta_state_size",
            "ta_state_save", "ta_state_load", "ta_batch_next", "ta_timing_begin", "ta_timing_end",
            "ta_grad_moments_static", "ta_static_last_error", "ta_test_expire_next_wait",
-           "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch", "ta_plan_pipeline",
+           "ta_power_iterate", "ta_set_curvature", "ta_plan_one_launch", "ta_plan_pipeline", "ta_plan_items",
            "ta_create_shard", "ta_shard_sweep", "ta_shard_apply", "ta_test_check_guards", "ta_path"]
 
 
@@ -114,6 +114,7 @@ def lib():
     L.ta_plan_one_launch.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_run), u32, C.POINTER(u32), C.POINTER(u32),
                                      C.POINTER(u32)]
     L.ta_plan_pipeline.argtypes = [C.POINTER(ta_segment), u32, u32, C.POINTER(ta_task), u64, C.POINTER(u64)]
+    L.ta_plan_items.argtypes = [C.POINTER(ta_segment), u32, u32, u32, C.POINTER(ta_run), u64, C.POINTER(u64), C.POINTER(u32)]
     L.ta_create_shard.argtypes = [C.POINTER(ta_segment), u32, u64, C.POINTER(ta_hparams), u64, u64, C.POINTER(vp)]
     L.ta_shard_sweep.argtypes = [vp, vp, vp, u64, u64, vp, vp]
     L.ta_shard_apply.argtypes = [vp, vp, vp, vp, vp, u32, vp]
@@ -340,6 +341,21 @@ def ta_plan_one_launch(table, warps):
     if rc != TA_OK:
         raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
     return [(r.begin, r.length, r.layer, r.warp) for r in out[:n.value]], used.value, rows.value
+
+
+def ta_plan_items(table, sm_count, topk=False):
+    """The work items of the multi-kernel pass: (items as a list of (begin, length, layer, warp, batch_in_one_layer), item_elems)."""
+    L = len(table)
+    segs = (ta_segment * max(L, 1))(*[ta_segment(int(o), int(n)) for o, n in table])
+    n, elems = C.c_uint64(), C.c_uint32()
+    rc = lib().ta_plan_items(segs, L, int(sm_count), 1 if topk else 0, None, 0, C.byref(n), C.byref(elems))
+    if rc != TA_OK and n.value == 0:
+        raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
+    out = (ta_run * max(1, n.value))()
+    rc = lib().ta_plan_items(segs, L, int(sm_count), 1 if topk else 0, out, n.value, C.byref(n), C.byref(elems))
+    if rc != TA_OK:
+        raise TriAccelError(rc, (lib().ta_last_error(None) or b"").decode())
+    return [(r.begin, r.length, r.layer, r.warp, r.reserved) for r in out[:n.value]], elems.value
 
 
 def ta_plan_pipeline(table, with_decisions=True):

@@ -172,6 +172,54 @@ uint32_t choose_item_elems(uint64_t n_params, int sm_count)
     return best;
 }
 
+// The work items of the multi-kernel pass: every layer (the part of it inside [range_lo, range_hi)) cut on a global
+// grid of item_elems elements, in buffer order; eight consecutive items make a batch, one per warp of a block.
+// topk: a layer of at least one full batch starts on a batch boundary, so that its batches hold one layer only and
+// can count their histogram in shared memory (the padding items are empty).  item_lo[l] is the first item of layer l,
+// batch_seg[b] the layer of a batch whose items all lie in one layer, else kMixedBatch.
+struct ItemPlan {
+    std::vector<ta::Item> items;
+    std::vector<uint32_t> item_lo, batch_seg;
+    bool too_many = false;
+};
+
+ItemPlan plan_items(const ta_segment *table, uint32_t L, uint32_t item_elems, bool topk, uint64_t range_lo, uint64_t range_hi)
+{
+    ItemPlan pl;
+    pl.item_lo.assign(L + 1, 0u);
+    std::vector<ta::Item> &items = pl.items;
+    for (uint32_t l = 0; l < L; ++l) {
+        pl.item_lo[l] = (uint32_t)items.size();
+        // a shard holds the part of every layer that lies inside its range (possibly nothing)
+        const uint64_t b = std::max<uint64_t>(table[l].offset, range_lo), e = std::min<uint64_t>(table[l].offset + table[l].length, range_hi);
+        if (e <= b) continue;
+        const uint64_t layer_items = (e - 1) / item_elems - b / item_elems + 1;
+        if (topk && layer_items >= (uint64_t)ta::kWarps && l > 0)
+            while (items.size() % ta::kWarps) items.push_back(ta::Item{b, 0u, l - 1});
+        pl.item_lo[l] = (uint32_t)items.size();
+        for (uint64_t p = b; p < e;) {
+            const uint64_t next = std::min(e, (p / item_elems + 1) * (uint64_t)item_elems);
+            items.push_back(ta::Item{p, (uint32_t)(next - p), l});
+            p = next;
+        }
+        if (items.size() > 0x7FFFFFFFull) { pl.too_many = true; return pl; }
+    }
+    pl.item_lo[L] = (uint32_t)items.size();
+    const uint32_t n_items = (uint32_t)items.size(), n_batches = (n_items + ta::kWarps - 1) / ta::kWarps;
+    pl.batch_seg.assign(n_batches, ta::kMixedBatch);
+    for (uint32_t bt = 0; bt < n_batches; ++bt) {
+        uint32_t seg = ta::kMixedBatch;
+        bool uniform = true;
+        for (uint32_t i = bt * ta::kWarps; i < std::min(n_items, (bt + 1) * ta::kWarps); ++i) {
+            if (items[i].len == 0) continue;
+            if (seg == ta::kMixedBatch) seg = items[i].seg;
+            else if (seg != items[i].seg) uniform = false;
+        }
+        pl.batch_seg[bt] = uniform ? seg : ta::kMixedBatch;
+    }
+    return pl;
+}
+
 int grid_for(const ta_handle *h)
 {
     const long long cap = (long long)h->sm_count * 8;
@@ -623,39 +671,18 @@ static int create_impl(const ta_segment *table, uint32_t L, uint64_t n_total, co
             run_plan = std::move(pl);
         }
     }
-    for (uint32_t l = 0; l < L && !h->fused_ok; ++l) {
-        item_lo[l] = (uint32_t)items.size();
-        // a shard holds the part of every layer that lies inside its range (possibly nothing)
-        const uint64_t b = std::max<uint64_t>(table[l].offset, h->range_lo), e = std::min<uint64_t>(table[l].offset + table[l].length, h->range_hi);
-        if (e <= b) continue;
-        // top-k: a layer of at least one full batch starts on a batch boundary, so that its batches hold one
-        // layer only and can count their histogram in shared memory (padding items are empty)
-        const uint64_t layer_items = (e - 1) / h->item_elems - b / h->item_elems + 1;
-        if (h->topk && layer_items >= (uint64_t)ta::kWarps && l > 0)
-            while (items.size() % ta::kWarps) items.push_back(ta::Item{b, 0u, l - 1});
-        item_lo[l] = (uint32_t)items.size();
-        for (uint64_t p = b; p < e;) {
-            const uint64_t next = std::min(e, (p / h->item_elems + 1) * (uint64_t)h->item_elems);
-            items.push_back(ta::Item{p, (uint32_t)(next - p), l});
-            p = next;
-        }
-        if (items.size() > 0x7FFFFFFFull) { snprintf(h->err, 256, "ta_create: too many work items"); return bail(TA_ERR_ARG); }
+    std::vector<uint32_t> batch_seg;
+    if (!h->fused_ok) {
+        ItemPlan ip = plan_items(table, L, h->item_elems, h->topk, h->range_lo, h->range_hi);
+        if (ip.too_many) { snprintf(h->err, 256, "ta_create: too many work items"); return bail(TA_ERR_ARG); }
+        items = std::move(ip.items);
+        item_lo = std::move(ip.item_lo);
+        batch_seg = std::move(ip.batch_seg);
     }
-    if (!h->fused_ok) item_lo[L] = (uint32_t)items.size();
     h->items_host = items;
     h->n_items = (uint32_t)items.size();
     h->n_batches = (h->n_items + ta::kWarps - 1) / ta::kWarps;
-    std::vector<uint32_t> batch_seg(h->n_batches, ta::kMixedBatch);
-    for (uint32_t bt = 0; bt < h->n_batches; ++bt) {
-        uint32_t seg = ta::kMixedBatch;
-        bool uniform = true;
-        for (uint32_t i = bt * ta::kWarps; i < std::min(h->n_items, (bt + 1) * ta::kWarps); ++i) {
-            if (items[i].len == 0) continue;
-            if (seg == ta::kMixedBatch) seg = items[i].seg;
-            else if (seg != items[i].seg) uniform = false;
-        }
-        batch_seg[bt] = uniform ? seg : ta::kMixedBatch;
-    }
+    if (h->fused_ok) batch_seg.assign(h->n_batches, ta::kMixedBatch);        // the one-launch path keeps no histogram
 
     DeviceBuffers &d = h->d;
     TA_TRY(dev_alloc(&d.items, items.size()));
@@ -903,6 +930,30 @@ int ta_plan_pipeline(const ta_segment *table, uint32_t L, uint32_t with_decision
     if (tasks.size() > cap || (!out && cap)) return fail(nullptr, TA_ERR_ARG, "ta_plan_pipeline: out is too small for the queues");
     for (size_t i = 0; i < tasks.size() && out; ++i)
         out[i] = ta_task{tasks[i].begin, tasks[i].len, tasks[i].seg_type & 0x3FFFFFFFu, tasks[i].seg_type >> 30, 0u};
+    return TA_OK;
+}
+
+int ta_plan_items(const ta_segment *table, uint32_t L, uint32_t sm_count, uint32_t topk, ta_run *out, uint64_t cap,
+                  uint64_t *n_items, uint32_t *item_elems)
+{
+    if (!table || L == 0 || !n_items || sm_count == 0) return fail(nullptr, TA_ERR_ARG, "ta_plan_items: table, L, sm_count and n_items are required");
+    uint64_t end = 0, n_params = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        if (table[l].length == 0 || table[l].length > 0xFFFFFFFEull)
+            return fail(nullptr, TA_ERR_ARG, "ta_plan_items: segment length out of range");
+        if (table[l].offset < end) return fail(nullptr, TA_ERR_ARG, "ta_plan_items: segments must be ascending and non-overlapping");
+        end = table[l].offset + table[l].length;
+        n_params += table[l].length;
+    }
+    const uint32_t elems = choose_item_elems(n_params, (int)sm_count);
+    const ItemPlan pl = plan_items(table, L, elems, topk != 0, 0, ~0ull);
+    if (pl.too_many) return fail(nullptr, TA_ERR_ARG, "ta_plan_items: too many work items");
+    *n_items = pl.items.size();
+    if (item_elems) *item_elems = elems;
+    if (pl.items.size() > cap || (!out && cap)) return fail(nullptr, TA_ERR_ARG, "ta_plan_items: out is too small for the items");
+    for (size_t i = 0; i < pl.items.size() && out; ++i)
+        out[i] = ta_run{pl.items[i].begin, pl.items[i].len, pl.items[i].seg, (uint32_t)(i % ta::kWarps),
+                        pl.batch_seg[i / ta::kWarps] == ta::kMixedBatch ? 0u : 1u};
     return TA_OK;
 }
 

@@ -310,3 +310,56 @@ def test_one_launch_plan_rejects_bad_tables():
         B.ta_plan_one_launch([(0, 10), (5, 10)], 64)          # overlapping
     with pytest.raises(B.TriAccelError):
         B.ta_plan_one_launch([(0, 0)], 64)                    # empty segment
+
+
+def _check_items(table, sm_count, topk):
+    items, elems = ta.ta_plan_items(table, sm_count, topk)
+    assert elems in (512, 1024, 2048, 4096, 8192, 16384)
+    pos = {l: off for l, (off, n) in enumerate(table)}
+    last_layer = 0
+    for i, (b, n, l, warp, one_layer) in enumerate(items):
+        assert warp == i % 8
+        if n == 0:
+            assert topk                      # padding in front of a layer that starts on a batch boundary
+            continue
+        assert l >= last_layer               # buffer order
+        last_layer = l
+        # consecutive pieces of the layer, cut on the global grid of `elems` elements
+        assert b == pos[l] and (b + n == table[l][0] + table[l][1] or (b + n) % elems == 0) and n <= elems
+        pos[l] += n
+    assert all(pos[l] == off + n for l, (off, n) in enumerate(table))       # every element exactly once
+    for bt in range(0, len(items), 8):
+        batch = items[bt:bt + 8]
+        layers = {l for _, n, l, _, _ in batch if n}
+        assert all(flag == (1 if len(layers) <= 1 else 0) for _, _, _, _, flag in batch)
+    if topk:
+        # a layer of at least eight items owns its batches
+        for l, (off, n) in enumerate(table):
+            mine = [i for i, it in enumerate(items) if it[2] == l and it[1]]
+            if len(mine) >= 8 and l > 0:
+                assert mine[0] % 8 == 0
+                assert all(items[i][4] == 1 for i in mine[: len(mine) // 8 * 8])
+    return items, elems
+
+
+def test_item_plan_of_the_multi_kernel_pass():
+    import numpy as np
+    from paper_2508_16905_b200 import workloads as W
+    items, elems = _check_items(W.get("resnet50_topk").table, 148, True)
+    assert elems == 4096 and len(items) < 8000
+    _check_items(W.get("resnet50_topk").table, 148, False)
+    items, elems = _check_items(W.get("gpt_1p3b").table, 148, False)
+    assert elems == 16384
+    rng = np.random.default_rng(11)
+    for trial in range(40):
+        L = int(rng.integers(1, 200))
+        lens = np.where(rng.random(L) < 0.6, rng.integers(1, 300, L), rng.integers(300, 300000, L))
+        gaps = rng.integers(0, 50, L) * (rng.random(L) < 0.5)
+        table, p = [], int(rng.integers(0, 9))
+        for n, gap in zip(lens, gaps):
+            p += int(gap)
+            table.append((p, int(n)))
+            p += int(n)
+        _check_items(table, int(rng.choice([1, 16, 148])), bool(trial % 2))
+    with pytest.raises(ta.TriAccelError):
+        ta.ta_plan_items([(0, 10), (5, 10)], 148, False)
