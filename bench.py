@@ -222,13 +222,25 @@ def measure(wl, hp, steps, warmup, dev, props, sample_clocks):
     curv = W.make_curvature(wl, dev)
     sets = []
     z = torch.empty(N, device=dev)
-    for r in range(R):
-        g = W.make_grads(wl, r + 1, dev)
+
+    def probe_products(t):
         hz = torch.empty(P * N, device=dev)
         for p in range(P):
-            ta.ta_probe(h, wl.probe_seed, r + 1, p, z)
+            ta.ta_probe(h, wl.probe_seed, t, p, z)
             torch.mul(curv, z, out=hz[p * N:(p + 1) * N])
-        sets.append((W.make_weights(wl, dev), g, hz, torch.zeros(N, dtype=torch.int16, device=dev)))
+        return hz
+
+    for r in range(R):
+        g = W.make_grads(wl, r + 1, dev)
+        sets.append((W.make_weights(wl, dev), g, probe_products(r + 1), torch.zeros(N, dtype=torch.int16, device=dev)))
+    # With one probe |z h| = |h| whatever the sign, so a buffer of probe products serves every step.  With several, the
+    # probes of step t are the ones the products must have been taken with, or the signs no longer cancel and |S| takes
+    # the values {0, 2D, 4D}: every step of the run then gets its own products (as a training loop would supply them),
+    # when the device has room for them.
+    total_steps = warmup + 2 * steps
+    per_step_hz = None
+    if P > 1 and total_steps * P * N * 4 <= 0.4 * props.total_memory:
+        per_step_hz = [probe_products(t) for t in range(1, total_steps + 1)]
     del z, curv
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
@@ -236,9 +248,12 @@ def measure(wl, hp, steps, warmup, dev, props, sample_clocks):
     import ctypes
     stream_arg = ctypes.c_void_p(stream.cuda_stream)
     ptrs = [tuple(ta.dev_ptr(x) for x in one) for one in sets]
+    hz_ptrs = [ta.dev_ptr(x) for x in per_step_hz] if per_step_hz is not None else None
 
     def one_step(t):
         w, g, hz, c = ptrs[t % R]
+        if hz_ptrs is not None:
+            hz = hz_ptrs[t - 1]
         ta.ta_step(h, w, g, hz, c, wl.probe_seed, t, stream_arg)
 
     t = 0
@@ -272,7 +287,10 @@ def measure(wl, hp, steps, warmup, dev, props, sample_clocks):
     stats, status = ta.ta_stats(h)
     assert status.skipped == 0, "a benchmark step was skipped (non-finite synthetic input?)"
     n_timed = max(1, n_timed)
-    out = {"ms_local": ms_local, "launches": int(launches), "path": path, "codes": [s.code for s in stats], "clocks": clocks, "R": R,
+    del per_step_hz
+    out = {"probe_signs": "one probe: any buffer serves" if P <= 1 else ("products taken with each step's own probes" if hz_ptrs is not None else
+                          "products of other steps' probes (no room for one buffer per step): |S| in {0, 2D, 4D}"),
+           "ms_local": ms_local, "launches": int(launches), "path": path, "codes": [s.code for s in stats], "clocks": clocks, "R": R,
            "bytes_in_per_set": bytes_in_per_set, "state_bytes": state_bytes, "l2_bytes": l2_bytes, "sets": sets,
            "phases": {"sweep": ms_sweep / n_timed, "decide_select": ms_decide / n_timed, "update": ms_update / n_timed}}
     ta.ta_destroy(h)
@@ -334,7 +352,8 @@ def describe(wl, m, steps, ms, peak, peak_kind, momentum=False, pipelined=False)
                "layers": len(wl.table), "algorithmic_bytes": ab["step"], "hbm_gbs_algorithmic": step_gbs,
                "frac_of_measured": step_gbs / peak, "frac_of_8tbs_nominal": step_gbs / 8000.0,
                "codes": {"fp16": codes.count(0), "bf16": codes.count(1), "fp32": codes.count(2)},
-               "launches_per_step": m["launches"] / steps, "path": m["path"], "l2": l2, "clocks": m["clocks"]}
+               "launches_per_step": m["launches"] / steps, "path": m["path"], "l2": l2, "probe_signs": m["probe_signs"],
+               "clocks": m["clocks"]}
     if wl.name in TARGETS:
         summary["target_frac_of_8tbs_nominal"] = TARGETS[wl.name]
         summary["target_met"] = summary["frac_of_8tbs_nominal"] >= TARGETS[wl.name]
@@ -442,7 +461,7 @@ def run_ours(args):
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "params": wl.num_params, "layers": len(wl.table), "grad_dtype": wl.grad_dtype,
                        "num_probes": P, "topk_ppm": wl.topk_ppm, "t_ctrl": wl.t_ctrl, "momentum": args.momentum,
-                       "weight_decay": args.weight_decay, "flags": flags, "parallelism": f"replicas x{world}", "l2": l2,
+                       "weight_decay": args.weight_decay, "flags": flags, "parallelism": f"replicas x{world}", "l2": l2, "probe_signs": m["probe_signs"],
                        "codes": {"fp16": codes.count(0), "bf16": codes.count(1), "fp32": codes.count(2)}},
             "hbm_gbs_algorithmic": roofline["step"]["achieved_gbs"],
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": m["launches"], "clocks": m["clocks"],
