@@ -1079,17 +1079,38 @@ __global__ void __launch_bounds__(kThreads) k_decide(const DecideArgs A)
     const float pivot_f = lo < hi ? A.p_piv[lo] : 0.f;
     const double pivot = (double)pivot_f;
     double n_local = 0.0;
-#pragma unroll 4
-    for (uint32_t i = lo + tid; i < hi; i += kThreads) {
-        const MomentSums m = rebase(A.p_s1[i], A.p_s2[i], (double)A.items[i].len, (double)A.p_piv[i], pivot);
-        s1 += m.s1;
-        s2 += m.s2;
-        n_local += (double)A.items[i].len;
-        bad += (double)A.p_bad[i];
-        if (A.has_hz) {
-            amax = max(amax, A.p_amax[i]);
-            amin = min(amin, A.p_amin[i]);
-            if (A.topk) sa += A.p_sa[i];
+    // Eight items per thread and trip, all their loads issued before the first is used (a layer of thousands of
+    // items is otherwise a chain of dependent trips to memory); each thread still adds its items in ascending order.
+    constexpr int kTrip = 8;
+    for (uint32_t i0 = lo + tid; i0 < hi; i0 += kThreads * kTrip) {
+        double x_s1[kTrip], x_s2[kTrip], x_sa[kTrip];
+        float x_piv[kTrip];
+        uint32_t x_len[kTrip], x_bad[kTrip], x_amax[kTrip], x_amin[kTrip];
+#pragma unroll
+        for (int k = 0; k < kTrip; ++k) {
+            const uint32_t i = i0 + (uint32_t)k * kThreads;
+            const bool in = i < hi;
+            x_s1[k] = in ? A.p_s1[i] : 0.0;
+            x_s2[k] = in ? A.p_s2[i] : 0.0;
+            x_piv[k] = in ? A.p_piv[i] : pivot_f;
+            x_len[k] = in ? A.items[i].len : 0u;
+            x_bad[k] = in ? A.p_bad[i] : 0u;
+            x_amax[k] = in && A.has_hz ? A.p_amax[i] : 0u;
+            x_amin[k] = in && A.has_hz ? A.p_amin[i] : 0xFFFFFFFFu;
+            x_sa[k] = in && A.has_hz && A.topk ? A.p_sa[i] : 0.0;
+        }
+#pragma unroll
+        for (int k = 0; k < kTrip; ++k) {
+            if (i0 + (uint32_t)k * kThreads < hi) {
+                const MomentSums m = rebase(x_s1[k], x_s2[k], (double)x_len[k], (double)x_piv[k], pivot);
+                s1 += m.s1;
+                s2 += m.s2;
+                n_local += (double)x_len[k];
+                bad += (double)x_bad[k];
+                amax = max(amax, x_amax[k]);
+                amin = min(amin, x_amin[k]);
+                sa += x_sa[k];
+            }
         }
     }
     s1 = block_sum(s1, red);
